@@ -1,0 +1,185 @@
+/*
+ * sifar.h - C ABI of the emulated synchronization-free all-reduce (one GPU).
+ *
+ * The operation (paper, Section 3.1 "Oneshot"): each of P tensor-parallel ranks
+ * holds a partial of n elements; every rank needs the element-wise sum.  Oneshot
+ * pulls all P partials and reduces locally, guarded by a TOP barrier (all
+ * partials produced before any pull: read-after-write) and a BOTTOM barrier (all
+ * pulls finished before a partial is overwritten: write-after-write).  The paper
+ * removes the bottom barrier by alternating two input buffers (Section 3.3,
+ * "dual buffering") and the cost of the top barrier by reading at once and
+ * validating afterwards (Sections 3.5 and 4.2, "speculative reduction").
+ *
+ * Here the P ranks are P equally laid out buffers in ONE GPU's memory, written by
+ * per-rank producer kernels on their own streams; one reducer kernel plays the
+ * pulling side.  There is no second GPU, no NVLink and no collective library.
+ * The paper's in-switch reduction ("redundant pull", Section 3.4) and multicast
+ * push are not part of this library.
+ *
+ * Result of every mode, exactly:  acc = widen(x_0[i]);  acc = acc + widen(x_r[i])
+ * for r = 1..P-1 in binary32, round-to-nearest-even;  out[i] = narrow(acc) with
+ * one RNE to the element type.
+ *
+ * All pointers named "device" are CUDA device pointers valid on the context's
+ * device; "stream" arguments are cudaStream_t passed as void* (NULL = the legacy
+ * default stream).  Functions return a sifar_status_t unless stated otherwise;
+ * no function throws, none synchronizes the device unless stated.
+ */
+#ifndef SIFAR_H
+#define SIFAR_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sifar_ctx sifar_ctx;   /* opaque, owned by the library */
+
+typedef enum { SIFAR_BF16 = 0, SIFAR_F32 = 1 } sifar_dtype;
+
+/*
+ * SIFAR_BARRIER_ONESHOT  baseline of Section 3.1: top barrier on P arrival flags,
+ *                        plain partials in ONE buffer per rank, bottom barrier
+ *                        (reducer CTAs all arrive, then P done flags are released;
+ *                        the rank's next producer waits on its done flag).
+ * SIFAR_DUALBUF          Section 3.3: two buffers per rank selected by the parity
+ *                        of the call number; top barrier kept, bottom barrier gone.
+ * SIFAR_SPECULATIVE      Sections 3.5 / 4.2 re-expressed for one GPU: the partial
+ *                        travels in 16-byte slots of 12 data bytes + a 4-byte tag
+ *                        equal to the call number; the reducer loads at once,
+ *                        accepts a slot iff its tag matches, and re-loads only the
+ *                        stale (rank, slot) pairs.  No flag, no barrier.
+ */
+typedef enum { SIFAR_BARRIER_ONESHOT = 0, SIFAR_DUALBUF = 1, SIFAR_SPECULATIVE = 2 } sifar_mode;
+
+typedef enum {
+    SIFAR_OK          =  0,
+    SIFAR_ERR_INVALID = -1,   /* bad argument; nothing was launched, call number unchanged */
+    SIFAR_ERR_NOMEM   = -2,
+    SIFAR_ERR_CUDA    = -3,   /* a CUDA call failed; sifar_last_error() has its text       */
+    SIFAR_ERR_TIMEOUT = -4,   /* a device-side wait ran out (sticky until sifar_reset)     */
+    SIFAR_ERR_EPOCH   = -5    /* call numbers exhausted, or a parity mismatch on the device */
+} sifar_status_t;
+
+enum { SIFAR_MAX_RANKS = 8 };
+
+/*
+ * Create a context for P ranks (1..8) of at most max_elems elements of `dtype`
+ * on the CURRENT device.  Allocates (cudaMalloc), once, per rank: two plain
+ * buffers, two slot buffers, and the shared flag / call-number / status words;
+ * everything zero-filled, so every tag starts as 0 = "never valid".
+ * Synchronizes the device.  Returns NULL on failure (see sifar_last_error()).
+ */
+sifar_ctx *sifar_create(int P, size_t max_elems, int dtype);
+
+/* Waits for the context's outstanding work, frees everything.  NULL is a no-op. */
+int sifar_destroy(sifar_ctx *ctx);
+
+/*
+ * Enqueue call number e = (calls so far) + 1 on `stream`: one reducer kernel, no
+ * allocation, no host synchronization.
+ *
+ *   rank_ptrs  host array of P device pointers, or NULL.
+ *              NULL: read the context's own rank buffers of this call (the buffers
+ *              sifar_rank_buffer() / sifar_pack() hand out).
+ *              non-NULL, mode BARRIER_ONESHOT: arbitrary caller buffers of n plain
+ *              elements each, 16-byte aligned, reusable every call; each rank's
+ *              stream must still announce them with sifar_arrive().
+ *              non-NULL, other modes: every pointer must equal the context's
+ *              buffer of this call, else SIFAR_ERR_INVALID.
+ *   out        device, n plain elements, 16-byte aligned, caller-owned, must not
+ *              overlap any rank buffer.  Valid once the kernel has finished
+ *              (stream order).
+ *   n          0 <= n <= max_elems.  n = 0 still consumes a call number.
+ *
+ * The reducer waits (barrier modes: for the arrival flags; speculative: per slot)
+ * until every rank's partial of THIS call number has been stored.  Producers may
+ * be enqueued on other streams before or after this call's kernel starts, but the
+ * host must have issued sifar_pack()/sifar_rank_buffer() for this call number
+ * before calling sifar_allreduce().  A wait that exceeds the time-out makes the
+ * kernel give up: the sticky status becomes SIFAR_ERR_TIMEOUT, `out` is undefined
+ * and later calls fail until sifar_reset().  Calls on one context must be
+ * enqueued on one stream (or otherwise serialized).
+ */
+int sifar_allreduce(sifar_ctx *ctx, const void *const *rank_ptrs, void *out, size_t n,
+                    int mode, void *stream);
+
+/*
+ * Same operation from HOST memory, synchronous: copies the P host partials
+ * (n plain elements each) to the device, packs them, reduces, copies the result
+ * to host_out and waits.  Uses staging buffers the context allocates on the first
+ * such call.  For end-to-end measurements and simple clients.
+ */
+int sifar_allreduce_host(sifar_ctx *ctx, const void *const *host_rank_ptrs, void *host_out,
+                         size_t n, int mode);
+
+/*
+ * Where, and with which tag, `rank` must store its partial for the NEXT call in
+ * `mode`.  *ptr: device buffer (plain elements for the barrier modes; 16-byte
+ * slots {12 data bytes, 4-byte little-endian tag} for SPECULATIVE, slot i holding
+ * elements [i*k, i*k+k), k = 6 for bf16 and 3 for fp32, a short last slot padded
+ * with zeros).  *epoch: the call number, i.e. the tag value.  Either may be NULL.
+ */
+int sifar_rank_buffer(sifar_ctx *ctx, int rank, int mode, void **ptr, unsigned *epoch);
+
+/*
+ * Library producer-side store path: enqueue on `stream` a kernel that moves n
+ * plain elements from `src` (device, 16-byte aligned) into the context's buffer
+ * of `rank` for the NEXT call: a copy followed by a release of the rank's arrival
+ * flag (barrier modes; BARRIER_ONESHOT first waits for the rank's done flag of
+ * the previous call), or tagged 16-byte slot stores and nothing else (SPECULATIVE).
+ */
+int sifar_pack(sifar_ctx *ctx, int rank, const void *src, size_t n, int mode, void *stream);
+
+/*
+ * Barrier modes with partials written by the caller's own kernels: enqueue on
+ * `stream` (after those kernels) the release of `rank`'s arrival flag for the
+ * NEXT call.
+ */
+int sifar_arrive(sifar_ctx *ctx, int rank, int mode, void *stream);
+
+/*
+ * BARRIER_ONESHOT only: enqueue on `stream` the producer-side half of the bottom
+ * barrier, a bounded wait until the reducer of the previous call has released
+ * `rank`'s done flag.  Enqueue it before the kernel that overwrites the buffer.
+ */
+int sifar_wait_writable(sifar_ctx *ctx, int rank, void *stream);
+
+/* Sticky device status (SIFAR_OK, SIFAR_ERR_TIMEOUT, SIFAR_ERR_EPOCH); reads a host-mapped word, no synchronization. */
+int sifar_status(sifar_ctx *ctx);
+
+/*
+ * Copies eight counters (synchronizes the device):
+ *   [0] calls completed        [1] calls in which at least one slot was re-loaded
+ *   [2] slot re-loads          [3] arrival-flag polls that found the flag not yet set
+ *   [4] waits that timed out   [5] current call number on the device   [6],[7] reserved
+ */
+int sifar_get_stats(sifar_ctx *ctx, unsigned long long out[8]);
+
+/* Limit of every device-side wait, in microseconds (default 200000). */
+int sifar_set_timeout_us(sifar_ctx *ctx, unsigned us);
+
+/* Waits for outstanding work on `stream`, zeroes tags, flags, counters and status; call number back to 0. */
+int sifar_reset(sifar_ctx *ctx, void *stream);
+
+/*
+ * Test hook: set the number of calls made so far (host and device).  Requires an
+ * idle context.  Call numbers are 32-bit; 0 is reserved, and the library refuses
+ * call number 2^32-1 and beyond with SIFAR_ERR_EPOCH until sifar_reset().
+ */
+int sifar_debug_set_epoch(sifar_ctx *ctx, unsigned calls_so_far);
+
+/* Geometry helpers (no device work). */
+size_t sifar_slot_count(int dtype, size_t n);          /* slots needed for n elements  */
+size_t sifar_algorithmic_bytes(int P, int dtype, size_t n, int mode);  /* bytes the method must move per call:
+                                                          P reads of the partial (plain or slots) + one write of
+                                                          out + the flag words of the mode */
+
+/* Text of the last error on the calling thread ("" if none). */
+const char *sifar_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SIFAR_H */

@@ -1,0 +1,144 @@
+"""Thin ctypes binding of ``libsifar.so``: same names as ``include/sifar.h``.
+
+Argument marshalling only.  Every step of the all-reduce runs in the CUDA
+library; there is no CPU fallback: if the library has not been built, the first
+call raises.  Device pointers are plain integers (``tensor.data_ptr()``), streams
+are ``torch.cuda.Stream().cuda_stream`` integers (0 = default stream).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+BF16, F32 = 0, 1
+BARRIER_ONESHOT, DUALBUF, SPECULATIVE = 0, 1, 2
+OK, ERR_INVALID, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT, ERR_EPOCH = 0, -1, -2, -3, -4, -5
+MODE_NAMES = {BARRIER_ONESHOT: "barrier_oneshot", DUALBUF: "dualbuf", SPECULATIVE: "speculative"}
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsifar.so")
+_lib = None
+
+
+class SifarError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"sifar error {code}: {text}")
+        self.code = code
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library (once).  Raises if it is missing: there is no other path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(
+                f"{_LIB_PATH} not found: build it with `python -m paper_2607_08973_b200.build`; "
+                "there is no CPU fallback")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, sz, ci, cu = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint
+        sig = {
+            "sifar_create": (vp, [ci, sz, ci]),
+            "sifar_destroy": (ci, [vp]),
+            "sifar_allreduce": (ci, [vp, vp, vp, sz, ci, vp]),
+            "sifar_allreduce_host": (ci, [vp, vp, vp, sz, ci]),
+            "sifar_rank_buffer": (ci, [vp, ci, ci, ctypes.POINTER(vp), ctypes.POINTER(cu)]),
+            "sifar_pack": (ci, [vp, ci, vp, sz, ci, vp]),
+            "sifar_arrive": (ci, [vp, ci, ci, vp]),
+            "sifar_wait_writable": (ci, [vp, ci, vp]),
+            "sifar_status": (ci, [vp]),
+            "sifar_get_stats": (ci, [vp, ctypes.POINTER(ctypes.c_ulonglong)]),
+            "sifar_set_timeout_us": (ci, [vp, cu]),
+            "sifar_reset": (ci, [vp, vp]),
+            "sifar_debug_set_epoch": (ci, [vp, cu]),
+            "sifar_slot_count": (sz, [ci, sz]),
+            "sifar_algorithmic_bytes": (sz, [ci, ci, sz, ci]),
+            "sifar_last_error": (ctypes.c_char_p, []),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def sifar_last_error() -> str:
+    return lib().sifar_last_error().decode()
+
+
+def _check(rc: int) -> int:
+    if rc != OK:
+        raise SifarError(rc, sifar_last_error())
+    return rc
+
+
+def sifar_create(P: int, max_elems: int, dtype: int) -> int:
+    h = lib().sifar_create(P, max_elems, dtype)
+    if not h:
+        raise SifarError(ERR_INVALID, sifar_last_error())
+    return h
+
+
+def sifar_destroy(ctx: int) -> int:
+    return _check(lib().sifar_destroy(ctx))
+
+
+def _ptr_array(ptrs):
+    if ptrs is None:
+        return None
+    return (ctypes.c_void_p * len(ptrs))(*ptrs)
+
+
+def sifar_allreduce(ctx: int, rank_ptrs, out: int, n: int, mode: int, stream: int = 0) -> int:
+    return _check(lib().sifar_allreduce(ctx, _ptr_array(rank_ptrs), out, n, mode, stream))
+
+
+def sifar_allreduce_host(ctx: int, host_rank_ptrs, host_out: int, n: int, mode: int) -> int:
+    return _check(lib().sifar_allreduce_host(ctx, _ptr_array(host_rank_ptrs), host_out, n, mode))
+
+
+def sifar_rank_buffer(ctx: int, rank: int, mode: int) -> tuple[int, int]:
+    p, e = ctypes.c_void_p(), ctypes.c_uint()
+    _check(lib().sifar_rank_buffer(ctx, rank, mode, ctypes.byref(p), ctypes.byref(e)))
+    return (p.value or 0), e.value
+
+
+def sifar_pack(ctx: int, rank: int, src: int, n: int, mode: int, stream: int = 0) -> int:
+    return _check(lib().sifar_pack(ctx, rank, src, n, mode, stream))
+
+
+def sifar_arrive(ctx: int, rank: int, mode: int, stream: int = 0) -> int:
+    return _check(lib().sifar_arrive(ctx, rank, mode, stream))
+
+
+def sifar_wait_writable(ctx: int, rank: int, stream: int = 0) -> int:
+    return _check(lib().sifar_wait_writable(ctx, rank, stream))
+
+
+def sifar_status(ctx: int) -> int:
+    return lib().sifar_status(ctx)
+
+
+def sifar_get_stats(ctx: int) -> dict:
+    buf = (ctypes.c_ulonglong * 8)()
+    _check(lib().sifar_get_stats(ctx, buf))
+    keys = ("calls", "calls_with_retry", "slot_reloads", "flag_polls", "timeouts", "epoch")
+    return {k: int(buf[i]) for i, k in enumerate(keys)}
+
+
+def sifar_set_timeout_us(ctx: int, us: int) -> int:
+    return _check(lib().sifar_set_timeout_us(ctx, us))
+
+
+def sifar_reset(ctx: int, stream: int = 0) -> int:
+    return _check(lib().sifar_reset(ctx, stream))
+
+
+def sifar_debug_set_epoch(ctx: int, calls_so_far: int) -> int:
+    return _check(lib().sifar_debug_set_epoch(ctx, calls_so_far))
+
+
+def sifar_slot_count(dtype: int, n: int) -> int:
+    return lib().sifar_slot_count(dtype, n)
+
+
+def sifar_algorithmic_bytes(P: int, dtype: int, n: int, mode: int) -> int:
+    return lib().sifar_algorithmic_bytes(P, dtype, n, mode)

@@ -1,0 +1,872 @@
+/*
+ * sifar_core.cu - context, producer-side store path and reducer kernels of the
+ * emulated oneshot all-reduce (sm_100a).
+ *
+ * Protocol per call number e (parity p = e & 1), after the paper's Sections 3.1,
+ * 3.3, 3.5 and 4.2, mapped onto one GPU:
+ *
+ *   BARRIER_ONESHOT  producer r : wait done[r] (bottom barrier, producer side);
+ *                                 plain stores into the rank's single buffer;
+ *                                 release arrive[p][r] = e.
+ *                    reducer    : poll arrive[p][0..P) == e (top barrier);
+ *                                 load, sum, store; all CTAs arrive on a counter,
+ *                                 the last one releases done[0..P) = e.
+ *   DUALBUF          producer r : plain stores into buffer p; release arrive.
+ *                    reducer    : top barrier; load, sum, store.
+ *   SPECULATIVE      producer r : one 16-byte store {12 B data, tag = e} per slot.
+ *                    reducer    : load all P slots at once, accept tag == e,
+ *                                 re-load only the stale ones (bounded); sum; store.
+ *
+ * The call number lives in device memory (DevState::epoch) and is read by every
+ * kernel at entry, so a replayed CUDA graph advances it without new arguments.
+ * Every wait is bounded by a time limit; on expiry the kernel records a sticky
+ * status and returns.
+ */
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "sifar_internal.cuh"
+
+namespace sifar {
+
+/* ------------------------------------------------------------------------ */
+/* errors                                                                    */
+/* ------------------------------------------------------------------------ */
+static thread_local char g_error[512] = "";
+
+void set_error(const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof g_error, fmt, ap);
+    va_end(ap);
+}
+
+int cuda_fail(cudaError_t e, const char *what)
+{
+    set_error("%s: %s", what, cudaGetErrorString(e));
+    return SIFAR_ERR_CUDA;
+}
+
+/* ------------------------------------------------------------------------ */
+/* kernel arguments                                                          */
+/* ------------------------------------------------------------------------ */
+struct ReduceArgs {
+    const uint4 *src[kMaxRanks];
+    void *out;
+    unsigned long long n;
+    DevState *st;
+    int *host_status;
+    unsigned long long timeout_ns;
+    uint32_t parity;
+    uint32_t check_parity;
+};
+
+struct PackArgs {
+    const void *src;
+    void *dst;
+    unsigned long long n;
+    DevState *st;
+    int *host_status;
+    unsigned long long timeout_ns;
+    uint32_t rank;
+    uint32_t parity;
+    uint32_t wait_delta;     /* 0: no bottom-barrier wait; d: wait for done[rank] >= e - d */
+};
+
+constexpr int kThreads = 256;
+
+/* ------------------------------------------------------------------------ */
+/* entry / exit of a reducer CTA                                             */
+/* ------------------------------------------------------------------------ */
+
+/* Bounded poll of a flag until it equals `want` (acquire).  Returns the number of failed polls, or -1 on time-out. */
+__device__ __forceinline__ int wait_flag_eq(const uint32_t *flag, uint32_t want, unsigned long long timeout_ns)
+{
+    int polls = 0;
+    unsigned long long t0 = 0;
+    while (ld_acquire_u32(flag) != want) {
+        ++polls;
+        unsigned long long now = globaltimer_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > timeout_ns) return -1;
+    }
+    return polls;
+}
+
+/* Same for "flag - base is in [0, 2^31)", i.e. flag has reached `base` (call numbers never wrap inside a context's life). */
+__device__ __forceinline__ int wait_flag_ge(const uint32_t *flag, uint32_t base, unsigned long long timeout_ns)
+{
+    int polls = 0;
+    unsigned long long t0 = 0;
+    while (ld_acquire_u32(flag) < base) {
+        ++polls;
+        unsigned long long now = globaltimer_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > timeout_ns) return -1;
+    }
+    return polls;
+}
+
+/*
+ * Completion of a reducer CTA, called by thread 0 after a __syncthreads().  The
+ * last CTA re-arms the counter, releases the done flags (bottom barrier, reducer
+ * side: every CTA has finished reading) and publishes the new call number.
+ */
+template <int MODE>
+__device__ __forceinline__ void reducer_finish(DevState *st, uint32_t e, int P)
+{
+    uint32_t n = gridDim.x;
+    uint32_t arrived = (n > 1) ? atom_add_acq_rel_u32(&st->cta_arrive, 1u) + 1u : 1u;
+    if (arrived == n) {
+        if (n > 1) st_relaxed_u32(&st->cta_arrive, 0u);
+        st->stats[kStatCalls] += 1ull;
+        if (MODE == SIFAR_SPECULATIVE && ld_relaxed_u32(&st->retry_epoch) == e)
+            st->stats[kStatCallsWithRetry] += 1ull;
+        if (MODE == SIFAR_BARRIER_ONESHOT)
+            for (int r = 0; r < P; ++r) st_release_u32(&st->done[r], e);
+        st_release_u32(&st->epoch, e);
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* rank-order accumulation                                                   */
+/* ------------------------------------------------------------------------ */
+template <int DT, int P>
+__device__ __forceinline__ uint32_t sum_word(const uint32_t (&w)[P])
+{
+    if (DT == SIFAR_BF16) {
+        float lo = bf16lo_to_f32(w[0]), hi = bf16hi_to_f32(w[0]);
+#pragma unroll
+        for (int r = 1; r < P; ++r) {
+            lo = __fadd_rn(lo, bf16lo_to_f32(w[r]));
+            hi = __fadd_rn(hi, bf16hi_to_f32(w[r]));
+        }
+        return f32x2_to_bf16x2(lo, hi);
+    } else {
+        float acc = __uint_as_float(w[0]);
+#pragma unroll
+        for (int r = 1; r < P; ++r) acc = __fadd_rn(acc, __uint_as_float(w[r]));
+        return __float_as_uint(acc);
+    }
+}
+
+template <int DT, int P>
+__device__ __forceinline__ uint4 sum_vec(const uint4 (&x)[P], bool with_w)
+{
+    uint32_t a[P], b[P], c[P], d[P];
+#pragma unroll
+    for (int r = 0; r < P; ++r) { a[r] = x[r].x; b[r] = x[r].y; c[r] = x[r].z; d[r] = x[r].w; }
+    uint4 o;
+    o.x = sum_word<DT, P>(a);
+    o.y = sum_word<DT, P>(b);
+    o.z = sum_word<DT, P>(c);
+    o.w = with_w ? sum_word<DT, P>(d) : 0u;
+    return o;
+}
+
+/* Vectors (plain) or slots (speculative) a thread keeps in flight per rank. */
+template <int P> struct Unroll { static constexpr int value = (P <= 2) ? 4 : (P <= 4) ? 2 : 1; };
+
+/* ------------------------------------------------------------------------ */
+/* reducer, barrier modes: plain partials behind arrival flags               */
+/* ------------------------------------------------------------------------ */
+template <int DT, int P, int MODE>
+__global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a)
+{
+    constexpr int U = Unroll<P>::value;
+    constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;       /* elements per 16-byte vector */
+    DevState *st = a.st;
+    __shared__ uint32_t s_epoch;
+
+    /* Top barrier (Section 3.1, phase 1): warp 0 polls the P arrival flags of this call. */
+    if (threadIdx.x < 32) {
+        const uint2 es = ld_relaxed_u32x2(&st->epoch);
+        const uint32_t e = es.x + 1u;
+        bool ok = (es.y == 0u);
+        if (ok && a.check_parity && (e & 1u) != a.parity) {
+            fail(st, a.host_status, SIFAR_ERR_EPOCH);
+            ok = false;
+        }
+        int polls = 0;
+        if (ok && threadIdx.x < P) {
+            polls = wait_flag_eq(&st->arrive[e & 1u][threadIdx.x], e, a.timeout_ns);
+            if (polls < 0) { fail(st, a.host_status, SIFAR_ERR_TIMEOUT); ok = false; polls = 0; }
+        }
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        polls = __reduce_add_sync(0xFFFFFFFFu, polls);
+        if (threadIdx.x == 0) {
+            s_epoch = ok ? e : 0u;
+            if (polls) atomicAdd(&st->stats[kStatFlagPolls], (unsigned long long)polls);
+        }
+    }
+    __syncthreads();
+    const uint32_t e = s_epoch;
+    if (e == 0u) return;
+
+    /* Pull and reduce (phase 2): P coalesced 16-byte loads per vector, all issued before the first add. */
+    const size_t nvec = (size_t)a.n / EPV;
+    uint4 *out = reinterpret_cast<uint4 *>(a.out);
+    const size_t stride = (size_t)gridDim.x * kThreads * U;
+    for (size_t base = (size_t)blockIdx.x * kThreads * U + threadIdx.x; base < nvec; base += stride) {
+        uint4 x[U][P];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t v = base + (size_t)u * kThreads;
+            if (v < nvec) {
+#pragma unroll
+                for (int r = 0; r < P; ++r) x[u][r] = ld_slot(a.src[r] + v);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t v = base + (size_t)u * kThreads;
+            if (v < nvec) out[v] = sum_vec<DT, P>(x[u], true);
+        }
+    }
+    /* Ragged tail: fewer than EPV elements, one per thread of CTA 0. */
+    const size_t tail0 = nvec * EPV;
+    if (blockIdx.x == 0 && tail0 + threadIdx.x < a.n) {
+        const size_t i = tail0 + threadIdx.x;
+        if (DT == SIFAR_BF16) {
+            uint32_t w[P];
+#pragma unroll
+            for (int r = 0; r < P; ++r)
+                w[r] = ld_relaxed_u16(reinterpret_cast<const uint16_t *>(a.src[r]) + i);
+            reinterpret_cast<uint16_t *>(a.out)[i] = (uint16_t)(sum_word<DT, P>(w) & 0xFFFFu);
+        } else {
+            uint32_t w[P];
+#pragma unroll
+            for (int r = 0; r < P; ++r)
+                w[r] = ld_relaxed_u32(reinterpret_cast<const uint32_t *>(a.src[r]) + i);
+            reinterpret_cast<uint32_t *>(a.out)[i] = sum_word<DT, P>(w);
+        }
+    }
+
+    /* Phase 3 (bottom barrier, baseline only) and publication of the call number. */
+    __syncthreads();
+    if (threadIdx.x == 0) reducer_finish<MODE>(st, e, P);
+}
+
+/* ------------------------------------------------------------------------ */
+/* reducer, speculative mode: tagged slots, per-slot validation and retry    */
+/* ------------------------------------------------------------------------ */
+template <int DT, int P>
+__global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
+{
+    constexpr int U = Unroll<P>::value;
+    constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;       /* elements per slot */
+    DevState *st = a.st;
+    const size_t nslots = ((size_t)a.n + EPS - 1) / EPS;
+
+    /* The call number is loaded together with the first slots: no dependent round trip before the data. */
+    const uint2 es = ld_relaxed_u32x2(&st->epoch);
+    uint32_t e = 0;
+    bool alive = true;
+    unsigned reloads = 0;
+
+    const size_t stride = (size_t)gridDim.x * kThreads * U;
+    for (size_t base = (size_t)blockIdx.x * kThreads * U + threadIdx.x; base < nslots && alive; base += stride) {
+        uint4 x[U][P];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t s = base + (size_t)u * kThreads;
+            if (s < nslots) {
+#pragma unroll
+                for (int r = 0; r < P; ++r) x[u][r] = ld_slot(a.src[r] + s);
+            }
+        }
+        if (e == 0u) {
+            e = es.x + 1u;
+            if (es.y != 0u) { alive = false; break; }
+            if (a.check_parity && (e & 1u) != a.parity) {
+                fail(st, a.host_status, SIFAR_ERR_EPOCH);
+                alive = false;
+                break;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t s = base + (size_t)u * kThreads;
+            if (s >= nslots) continue;
+            /* Validation (Section 4.2): a slot counts iff it carries this call's tag. */
+            uint32_t stale = 0;
+#pragma unroll
+            for (int r = 0; r < P; ++r) stale |= (uint32_t)(x[u][r].w != e) << r;
+            if (stale) {
+                /* Mis-speculation: re-load only the stale ranks of this slot, with back-off, until the time limit. */
+                const unsigned long long t0 = globaltimer_ns();
+                unsigned spins = 0;
+                do {
+#pragma unroll
+                    for (int r = 0; r < P; ++r) {
+                        if (stale & (1u << r)) {
+                            x[u][r] = ld_slot(a.src[r] + s);
+                            ++reloads;
+                            if (x[u][r].w == e) stale &= ~(1u << r);
+                        }
+                    }
+                    if (stale) {
+                        if (globaltimer_ns() - t0 > a.timeout_ns) {
+                            fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+                            alive = false;
+                            break;
+                        }
+                        if (++spins > 8) __nanosleep(spins > 64 ? 200 : 40);
+                    }
+                } while (stale);
+                if (!alive) break;
+            }
+            const uint4 o = sum_vec<DT, P>(x[u], false);
+            const size_t i0 = s * EPS;
+            if (i0 + EPS <= a.n) {
+                uint32_t *dst = reinterpret_cast<uint32_t *>(a.out) + s * 3;
+                dst[0] = o.x; dst[1] = o.y; dst[2] = o.z;
+            } else if (DT == SIFAR_BF16) {
+                uint16_t *dst = reinterpret_cast<uint16_t *>(a.out) + i0;
+                const uint32_t w[3] = {o.x, o.y, o.z};
+                for (int k = 0; k < EPS && i0 + k < a.n; ++k)
+                    dst[k] = (uint16_t)((w[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu);
+            } else {
+                uint32_t *dst = reinterpret_cast<uint32_t *>(a.out) + i0;
+                const uint32_t w[3] = {o.x, o.y, o.z};
+                for (int k = 0; k < EPS && i0 + k < a.n; ++k) dst[k] = w[k];
+            }
+        }
+    }
+
+    /* Threads without a slot still need the call number for the completion step. */
+    if (e == 0u && alive) {
+        e = es.x + 1u;
+        if (es.y != 0u) alive = false;
+        else if (a.check_parity && (e & 1u) != a.parity) { fail(st, a.host_status, SIFAR_ERR_EPOCH); alive = false; }
+    }
+
+    /* Mis-speculation statistics: one atomic per warp that re-loaded anything. */
+    const unsigned warp_reloads = __reduce_add_sync(0xFFFFFFFFu, reloads);
+    if (warp_reloads && (threadIdx.x & 31) == 0) {
+        atomicAdd(&st->stats[kStatSlotReloads], (unsigned long long)warp_reloads);
+        st_relaxed_u32(&st->retry_epoch, e);
+    }
+    const int all_alive = __syncthreads_and(alive);
+    if (!all_alive) return;
+    if (threadIdx.x == 0) reducer_finish<SIFAR_SPECULATIVE>(st, e, P);
+}
+
+/* ------------------------------------------------------------------------ */
+/* producer-side store path                                                  */
+/* ------------------------------------------------------------------------ */
+template <int DT, int MODE>
+__global__ void __launch_bounds__(kThreads) k_pack(const PackArgs a)
+{
+    DevState *st = a.st;
+    __shared__ uint32_t s_epoch;
+    if (threadIdx.x == 0) {
+        const uint2 es = ld_relaxed_u32x2(&st->epoch);
+        uint32_t e = es.x + 1u;
+        bool ok = (es.y == 0u);
+        if (ok && MODE != SIFAR_BARRIER_ONESHOT && (e & 1u) != a.parity) {
+            fail(st, a.host_status, SIFAR_ERR_EPOCH);
+            ok = false;
+        }
+        /* Bottom barrier, producer side: the previous reader of this single buffer must be done. */
+        if (ok && MODE == SIFAR_BARRIER_ONESHOT && a.wait_delta) {
+            if (wait_flag_ge(&st->done[a.rank], e - a.wait_delta, a.timeout_ns) < 0) {
+                fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+                ok = false;
+            }
+        }
+        s_epoch = ok ? e : 0u;
+    }
+    __syncthreads();
+    const uint32_t e = s_epoch;
+    if (e == 0u) return;
+
+    const size_t tid = (size_t)blockIdx.x * kThreads + threadIdx.x;
+    const size_t nthreads = (size_t)gridDim.x * kThreads;
+    if (MODE != SIFAR_SPECULATIVE) {
+        constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
+        const size_t nvec = (size_t)a.n / EPV;
+        const uint4 *src = reinterpret_cast<const uint4 *>(a.src);
+        uint4 *dst = reinterpret_cast<uint4 *>(a.dst);
+        for (size_t v = tid; v < nvec; v += nthreads) st_slot(dst + v, src[v]);
+        const size_t i = nvec * EPV + threadIdx.x;
+        if (blockIdx.x == 0 && i < a.n) {
+            if (DT == SIFAR_BF16)
+                reinterpret_cast<uint16_t *>(a.dst)[i] = reinterpret_cast<const uint16_t *>(a.src)[i];
+            else
+                reinterpret_cast<uint32_t *>(a.dst)[i] = reinterpret_cast<const uint32_t *>(a.src)[i];
+        }
+        signal_arrival(&st->pack_count[a.rank], gridDim.x, &st->arrive[e & 1u][a.rank], e);
+    } else {
+        constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;
+        const size_t nslots = ((size_t)a.n + EPS - 1) / EPS;
+        uint4 *slots = reinterpret_cast<uint4 *>(a.dst);
+        const uint32_t *src32 = reinterpret_cast<const uint32_t *>(a.src);
+        for (size_t s = tid; s < nslots; s += nthreads) {
+            uint32_t w[3] = {0u, 0u, 0u};
+            const size_t i0 = s * EPS;
+            if (i0 + EPS <= a.n) {
+                w[0] = src32[s * 3]; w[1] = src32[s * 3 + 1]; w[2] = src32[s * 3 + 2];
+            } else if (DT == SIFAR_BF16) {
+                const uint16_t *src16 = reinterpret_cast<const uint16_t *>(a.src);
+                for (int k = 0; k < EPS && i0 + k < a.n; ++k)
+                    w[k >> 1] |= (uint32_t)src16[i0 + k] << ((k & 1) * 16);
+            } else {
+                for (int k = 0; k < EPS && i0 + k < a.n; ++k) w[k] = src32[i0 + k];
+            }
+            store_slot(slots, s, w[0], w[1], w[2], e);
+        }
+    }
+}
+
+/* Release of one rank's arrival flag after caller-written plain partials. */
+__global__ void k_arrive(DevState *st, uint32_t rank)
+{
+    const uint2 es = ld_relaxed_u32x2(&st->epoch);
+    if (es.y != 0u) return;
+    const uint32_t e = es.x + 1u;
+    __threadfence();
+    st_release_u32(&st->arrive[e & 1u][rank], e);
+}
+
+/* Producer-side half of the bottom barrier as a kernel of its own. */
+__global__ void k_wait_writable(DevState *st, int *host_status, uint32_t rank, uint32_t wait_delta,
+                                unsigned long long timeout_ns)
+{
+    const uint2 es = ld_relaxed_u32x2(&st->epoch);
+    if (es.y != 0u) return;
+    const uint32_t e = es.x + 1u;
+    if (wait_flag_ge(&st->done[rank], e - wait_delta, timeout_ns) < 0) fail(st, host_status, SIFAR_ERR_TIMEOUT);
+}
+
+/* n = 0: nothing to move, the call number still advances. */
+__global__ void k_empty_call(DevState *st, int mode, int P)
+{
+    const uint2 es = ld_relaxed_u32x2(&st->epoch);
+    if (es.y != 0u) return;
+    const uint32_t e = es.x + 1u;
+    st->stats[kStatCalls] += 1ull;
+    if (mode == SIFAR_BARRIER_ONESHOT)
+        for (int r = 0; r < P; ++r) st_release_u32(&st->done[r], e);
+    st_release_u32(&st->epoch, e);
+}
+
+__global__ void k_set_epoch(DevState *st, uint32_t e) { st->epoch = e; }
+
+/* ------------------------------------------------------------------------ */
+/* launch geometry                                                           */
+/* ------------------------------------------------------------------------ */
+static int reduce_grid(const sifar_ctx *ctx, size_t units, int per_thread)
+{
+    const size_t per_cta = (size_t)kThreads * per_thread;
+    size_t ctas = (units + per_cta - 1) / per_cta;
+    const size_t cap = (size_t)ctx->sm_count * 4;          /* 4 CTAs of 256 threads per SM: one wave */
+    if (ctas > cap) ctas = cap;
+    if (ctas < 1) ctas = 1;
+    return (int)ctas;
+}
+
+template <int DT, int P>
+static cudaError_t launch_reduce_p(int mode, int grid, cudaStream_t s, const ReduceArgs &a)
+{
+    switch (mode) {
+    case SIFAR_BARRIER_ONESHOT: k_reduce_plain<DT, P, SIFAR_BARRIER_ONESHOT><<<grid, kThreads, 0, s>>>(a); break;
+    case SIFAR_DUALBUF:         k_reduce_plain<DT, P, SIFAR_DUALBUF><<<grid, kThreads, 0, s>>>(a); break;
+    default:                    k_reduce_spec<DT, P><<<grid, kThreads, 0, s>>>(a); break;
+    }
+    return cudaGetLastError();
+}
+
+template <int DT>
+static cudaError_t launch_reduce_dt(int P, int mode, int grid, cudaStream_t s, const ReduceArgs &a)
+{
+    switch (P) {
+    case 1: return launch_reduce_p<DT, 1>(mode, grid, s, a);
+    case 2: return launch_reduce_p<DT, 2>(mode, grid, s, a);
+    case 3: return launch_reduce_p<DT, 3>(mode, grid, s, a);
+    case 4: return launch_reduce_p<DT, 4>(mode, grid, s, a);
+    case 5: return launch_reduce_p<DT, 5>(mode, grid, s, a);
+    case 6: return launch_reduce_p<DT, 6>(mode, grid, s, a);
+    case 7: return launch_reduce_p<DT, 7>(mode, grid, s, a);
+    default: return launch_reduce_p<DT, 8>(mode, grid, s, a);
+    }
+}
+
+static int unroll_for(int P) { return P <= 2 ? 4 : P <= 4 ? 2 : 1; }
+
+int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
+{
+    if (rl.n == 0) {
+        k_empty_call<<<1, 1, 0, stream>>>(ctx->d_state, rl.mode, ctx->P);
+        SIFAR_CUDA(cudaGetLastError());
+        return SIFAR_OK;
+    }
+    ReduceArgs a;
+    memset(&a, 0, sizeof a);
+    for (int r = 0; r < ctx->P; ++r) a.src[r] = reinterpret_cast<const uint4 *>(rl.src[r]);
+    a.out = rl.out;
+    a.n = rl.n;
+    a.st = ctx->d_state;
+    a.host_status = ctx->d_status_alias;
+    a.timeout_ns = ctx->timeout_ns;
+    a.parity = rl.parity;
+    a.check_parity = (rl.mode != SIFAR_BARRIER_ONESHOT);
+    size_t units = (rl.mode == SIFAR_SPECULATIVE) ? slots_for(ctx->dtype, rl.n)
+                                                  : (rl.n * elem_size(ctx->dtype) + 15) / 16;
+    const int grid = reduce_grid(ctx, units, unroll_for(ctx->P));
+    cudaError_t err = (ctx->dtype == SIFAR_BF16)
+        ? launch_reduce_dt<SIFAR_BF16>(ctx->P, rl.mode, grid, stream, a)
+        : launch_reduce_dt<SIFAR_F32>(ctx->P, rl.mode, grid, stream, a);
+    SIFAR_CUDA(err);
+    return SIFAR_OK;
+}
+
+template <int DT>
+static cudaError_t launch_pack_dt(int mode, int grid, cudaStream_t s, const PackArgs &a)
+{
+    switch (mode) {
+    case SIFAR_BARRIER_ONESHOT: k_pack<DT, SIFAR_BARRIER_ONESHOT><<<grid, kThreads, 0, s>>>(a); break;
+    case SIFAR_DUALBUF:         k_pack<DT, SIFAR_DUALBUF><<<grid, kThreads, 0, s>>>(a); break;
+    default:                    k_pack<DT, SIFAR_SPECULATIVE><<<grid, kThreads, 0, s>>>(a); break;
+    }
+    return cudaGetLastError();
+}
+
+}  /* namespace sifar */
+
+using namespace sifar;
+
+/* ------------------------------------------------------------------------ */
+/* C ABI                                                                     */
+/* ------------------------------------------------------------------------ */
+static bool valid_mode(int m) { return m == SIFAR_BARRIER_ONESHOT || m == SIFAR_DUALBUF || m == SIFAR_SPECULATIVE; }
+static bool valid_dtype(int d) { return d == SIFAR_BF16 || d == SIFAR_F32; }
+static size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+extern "C" const char *sifar_last_error(void) { return g_error; }
+
+extern "C" size_t sifar_slot_count(int dtype, size_t n)
+{
+    return valid_dtype(dtype) ? slots_for(dtype, n) : 0;
+}
+
+extern "C" size_t sifar_algorithmic_bytes(int P, int dtype, size_t n, int mode)
+{
+    if (!valid_dtype(dtype) || !valid_mode(mode) || P < 1) return 0;
+    const size_t payload = n * elem_size(dtype);
+    const size_t per_rank = (mode == SIFAR_SPECULATIVE) ? slots_for(dtype, n) * 16 : payload;
+    size_t flags = 0;
+    if (mode != SIFAR_SPECULATIVE) flags += (size_t)P * 4;          /* arrival flags */
+    if (mode == SIFAR_BARRIER_ONESHOT) flags += (size_t)P * 4;      /* done flags    */
+    return (size_t)P * per_rank + payload + flags;
+}
+
+extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
+{
+    g_error[0] = 0;
+    if (P < 1 || P > kMaxRanks || max_elems == 0 || !valid_dtype(dtype)) {
+        set_error("sifar_create: need 1 <= P <= %d, max_elems > 0, dtype in {0,1}", kMaxRanks);
+        return nullptr;
+    }
+    if (max_elems > ((size_t)1 << 31)) {
+        set_error("sifar_create: max_elems above 2^31 is not supported");
+        return nullptr;
+    }
+    sifar_ctx *c = new (std::nothrow) sifar_ctx();
+    if (!c) { set_error("sifar_create: out of host memory"); return nullptr; }
+    memset(c, 0, sizeof *c);
+    c->P = P; c->dtype = dtype; c->max_elems = max_elems;
+    c->timeout_ns = 200000ull * 1000ull;
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+    c->plain_stride = round_up(max_elems * elem_size(dtype), 256);
+    c->slot_stride = round_up(slots_for(dtype, max_elems) * 16, 256);
+    const size_t plain_bytes = c->plain_stride * 2 * P, slot_bytes = c->slot_stride * 2 * P;
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_plain, plain_bytes);
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_slots, slot_bytes);
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_state, sizeof(DevState));
+    if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->h_status, sizeof(int), cudaHostAllocMapped);
+    if (e == cudaSuccess) { *c->h_status = 0; e = cudaHostGetDevicePointer((void **)&c->d_status_alias, (void *)c->h_status, 0); }
+    if (e == cudaSuccess) e = cudaMemset(c->d_plain, 0, plain_bytes);
+    if (e == cudaSuccess) e = cudaMemset(c->d_slots, 0, slot_bytes);
+    if (e == cudaSuccess) e = cudaMemset(c->d_state, 0, sizeof(DevState));
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->host_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        set_error("sifar_create: %s", cudaGetErrorString(e));
+        const bool nomem = (e == cudaErrorMemoryAllocation);
+        cudaGetLastError();
+        if (c->d_plain) cudaFree(c->d_plain);
+        if (c->d_slots) cudaFree(c->d_slots);
+        if (c->d_state) cudaFree(c->d_state);
+        if (c->h_status) cudaFreeHost((void *)c->h_status);
+        if (c->host_stream) cudaStreamDestroy(c->host_stream);
+        delete c;
+        (void)nomem;
+        return nullptr;
+    }
+    return c;
+}
+
+extern "C" int sifar_destroy(sifar_ctx *c)
+{
+    if (!c) return SIFAR_OK;
+    cudaSetDevice(c->device);
+    cudaError_t e = cudaDeviceSynchronize();
+    cudaFree(c->d_plain);
+    cudaFree(c->d_slots);
+    cudaFree(c->d_state);
+    if (c->d_stage_in) cudaFree(c->d_stage_in);
+    if (c->d_stage_out) cudaFree(c->d_stage_out);
+    cudaFreeHost((void *)c->h_status);
+    cudaStreamDestroy(c->host_stream);
+    delete c;
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+    return SIFAR_OK;
+}
+
+static int check_live(sifar_ctx *c, const char *fn)
+{
+    if (!c) { set_error("%s: NULL context", fn); return SIFAR_ERR_INVALID; }
+    const int s = *c->h_status;
+    if (s != 0) { set_error("%s: context carries device status %d; call sifar_reset", fn, s); return s; }
+    return SIFAR_OK;
+}
+
+static int next_epoch(sifar_ctx *c, const char *fn, uint32_t *e)
+{
+    if (c->h_epoch >= kEpochLimit) {
+        set_error("%s: call numbers exhausted; call sifar_reset", fn);
+        return SIFAR_ERR_EPOCH;
+    }
+    *e = c->h_epoch + 1u;
+    return SIFAR_OK;
+}
+
+static const void *ctx_buffer(const sifar_ctx *c, int mode, uint32_t e, int r)
+{
+    if (mode == SIFAR_BARRIER_ONESHOT) return c->plain_buf(0, r);
+    if (mode == SIFAR_DUALBUF) return c->plain_buf((int)(e & 1u), r);
+    return c->slot_buf((int)(e & 1u), r);
+}
+
+static size_t ctx_buffer_bytes(const sifar_ctx *c, int mode, size_t n)
+{
+    return mode == SIFAR_SPECULATIVE ? slots_for(c->dtype, n) * 16 : n * elem_size(c->dtype);
+}
+
+static bool overlaps(const void *a, size_t na, const void *b, size_t nb)
+{
+    const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+    return x < y + nb && y < x + na;
+}
+
+extern "C" int sifar_allreduce(sifar_ctx *c, const void *const *rank_ptrs, void *out, size_t n, int mode,
+                               void *stream)
+{
+    int rc = check_live(c, "sifar_allreduce");
+    if (rc) return rc;
+    if (!valid_mode(mode)) { set_error("sifar_allreduce: unknown mode %d", mode); return SIFAR_ERR_INVALID; }
+    if (n > c->max_elems) { set_error("sifar_allreduce: n exceeds max_elems"); return SIFAR_ERR_INVALID; }
+    if (n > 0 && (!out || ((uintptr_t)out & 15u))) {
+        set_error("sifar_allreduce: out must be a 16-byte aligned device pointer");
+        return SIFAR_ERR_INVALID;
+    }
+    uint32_t e;
+    if ((rc = next_epoch(c, "sifar_allreduce", &e))) return rc;
+
+    ReduceLaunch rl;
+    memset(&rl, 0, sizeof rl);
+    const size_t in_bytes = ctx_buffer_bytes(c, mode, n), out_bytes = n * elem_size(c->dtype);
+    for (int r = 0; r < c->P; ++r) {
+        const void *own = ctx_buffer(c, mode, e, r);
+        const void *p = own;
+        if (rank_ptrs) {
+            p = rank_ptrs[r];
+            if (mode != SIFAR_BARRIER_ONESHOT && p != own) {
+                set_error("sifar_allreduce: rank_ptrs[%d] is not the context's buffer of this call", r);
+                return SIFAR_ERR_INVALID;
+            }
+            if (!p || ((uintptr_t)p & 15u)) {
+                set_error("sifar_allreduce: rank_ptrs[%d] must be a 16-byte aligned device pointer", r);
+                return SIFAR_ERR_INVALID;
+            }
+        }
+        if (n > 0 && overlaps(out, out_bytes, p, in_bytes)) {
+            set_error("sifar_allreduce: out overlaps the buffer of rank %d", r);
+            return SIFAR_ERR_INVALID;
+        }
+        rl.src[r] = p;
+    }
+    rl.out = out; rl.n = n; rl.mode = mode; rl.parity = e & 1u;
+    rc = launch_reduce(c, rl, (cudaStream_t)stream);
+    if (rc) return rc;
+    c->h_epoch = e;
+    if (mode == SIFAR_BARRIER_ONESHOT) c->last_mode0_epoch = e;
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_rank_buffer(sifar_ctx *c, int rank, int mode, void **ptr, unsigned *epoch)
+{
+    if (!c) { set_error("sifar_rank_buffer: NULL context"); return SIFAR_ERR_INVALID; }
+    if (rank < 0 || rank >= c->P || !valid_mode(mode)) {
+        set_error("sifar_rank_buffer: bad rank or mode");
+        return SIFAR_ERR_INVALID;
+    }
+    uint32_t e;
+    int rc = next_epoch(c, "sifar_rank_buffer", &e);
+    if (rc) return rc;
+    if (ptr) *ptr = const_cast<void *>(ctx_buffer(c, mode, e, rank));
+    if (epoch) *epoch = e;
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_pack(sifar_ctx *c, int rank, const void *src, size_t n, int mode, void *stream)
+{
+    int rc = check_live(c, "sifar_pack");
+    if (rc) return rc;
+    if (rank < 0 || rank >= c->P || !valid_mode(mode) || n > c->max_elems) {
+        set_error("sifar_pack: bad rank, mode or n");
+        return SIFAR_ERR_INVALID;
+    }
+    if (n > 0 && (!src || ((uintptr_t)src & 15u))) {
+        set_error("sifar_pack: src must be a 16-byte aligned device pointer");
+        return SIFAR_ERR_INVALID;
+    }
+    uint32_t e;
+    if ((rc = next_epoch(c, "sifar_pack", &e))) return rc;
+    PackArgs a;
+    memset(&a, 0, sizeof a);
+    a.src = src;
+    a.dst = const_cast<void *>(ctx_buffer(c, mode, e, rank));
+    a.n = n;
+    a.st = c->d_state;
+    a.host_status = c->d_status_alias;
+    a.timeout_ns = c->timeout_ns;
+    a.rank = (uint32_t)rank;
+    a.parity = e & 1u;
+    a.wait_delta = (mode == SIFAR_BARRIER_ONESHOT && c->last_mode0_epoch) ? e - c->last_mode0_epoch : 0u;
+    const size_t units = (mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, n) : (n * elem_size(c->dtype) + 15) / 16;
+    size_t grid = (units + kThreads - 1) / kThreads;
+    const size_t cap = (size_t)c->sm_count * 2;
+    if (grid > cap) grid = cap;
+    if (grid < 1) grid = 1;
+    cudaError_t err = (c->dtype == SIFAR_BF16) ? launch_pack_dt<SIFAR_BF16>(mode, (int)grid, (cudaStream_t)stream, a)
+                                               : launch_pack_dt<SIFAR_F32>(mode, (int)grid, (cudaStream_t)stream, a);
+    SIFAR_CUDA(err);
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_arrive(sifar_ctx *c, int rank, int mode, void *stream)
+{
+    int rc = check_live(c, "sifar_arrive");
+    if (rc) return rc;
+    if (rank < 0 || rank >= c->P || (mode != SIFAR_BARRIER_ONESHOT && mode != SIFAR_DUALBUF)) {
+        set_error("sifar_arrive: bad rank, or a mode without arrival flags");
+        return SIFAR_ERR_INVALID;
+    }
+    k_arrive<<<1, 1, 0, (cudaStream_t)stream>>>(c->d_state, (uint32_t)rank);
+    SIFAR_CUDA(cudaGetLastError());
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_wait_writable(sifar_ctx *c, int rank, void *stream)
+{
+    int rc = check_live(c, "sifar_wait_writable");
+    if (rc) return rc;
+    if (rank < 0 || rank >= c->P) { set_error("sifar_wait_writable: bad rank"); return SIFAR_ERR_INVALID; }
+    if (!c->last_mode0_epoch) return SIFAR_OK;      /* nothing has read the buffer yet */
+    const uint32_t delta = c->h_epoch + 1u - c->last_mode0_epoch;
+    k_wait_writable<<<1, 1, 0, (cudaStream_t)stream>>>(c->d_state, c->d_status_alias, (uint32_t)rank, delta,
+                                                       c->timeout_ns);
+    SIFAR_CUDA(cudaGetLastError());
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_status(sifar_ctx *c)
+{
+    if (!c) { set_error("sifar_status: NULL context"); return SIFAR_ERR_INVALID; }
+    return *c->h_status;
+}
+
+extern "C" int sifar_get_stats(sifar_ctx *c, unsigned long long out[8])
+{
+    if (!c || !out) { set_error("sifar_get_stats: NULL argument"); return SIFAR_ERR_INVALID; }
+    DevState h;
+    SIFAR_CUDA(cudaDeviceSynchronize());
+    SIFAR_CUDA(cudaMemcpy(&h, c->d_state, sizeof h, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < 5; ++i) out[i] = h.stats[i];
+    out[5] = h.epoch; out[6] = 0; out[7] = 0;
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_set_timeout_us(sifar_ctx *c, unsigned us)
+{
+    if (!c || us == 0) { set_error("sifar_set_timeout_us: NULL context or zero"); return SIFAR_ERR_INVALID; }
+    c->timeout_ns = (unsigned long long)us * 1000ull;
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_reset(sifar_ctx *c, void *stream)
+{
+    if (!c) { set_error("sifar_reset: NULL context"); return SIFAR_ERR_INVALID; }
+    cudaStream_t s = (cudaStream_t)stream;
+    SIFAR_CUDA(cudaDeviceSynchronize());
+    SIFAR_CUDA(cudaMemsetAsync(c->d_slots, 0, c->slot_stride * 2 * c->P, s));
+    SIFAR_CUDA(cudaMemsetAsync(c->d_state, 0, sizeof(DevState), s));
+    SIFAR_CUDA(cudaStreamSynchronize(s));
+    *c->h_status = 0;
+    c->h_epoch = 0;
+    c->last_mode0_epoch = 0;
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_debug_set_epoch(sifar_ctx *c, unsigned calls_so_far)
+{
+    if (!c) { set_error("sifar_debug_set_epoch: NULL context"); return SIFAR_ERR_INVALID; }
+    SIFAR_CUDA(cudaDeviceSynchronize());
+    k_set_epoch<<<1, 1>>>(c->d_state, calls_so_far);
+    SIFAR_CUDA(cudaGetLastError());
+    SIFAR_CUDA(cudaDeviceSynchronize());
+    c->h_epoch = calls_so_far;
+    c->last_mode0_epoch = 0;
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_allreduce_host(sifar_ctx *c, const void *const *host_rank_ptrs, void *host_out, size_t n,
+                                    int mode)
+{
+    int rc = check_live(c, "sifar_allreduce_host");
+    if (rc) return rc;
+    if (!valid_mode(mode) || n > c->max_elems || !host_rank_ptrs || (n > 0 && !host_out)) {
+        set_error("sifar_allreduce_host: bad mode, n or pointer");
+        return SIFAR_ERR_INVALID;
+    }
+    const size_t stride = c->plain_stride;
+    if (!c->d_stage_in) {
+        cudaError_t e = cudaMalloc(&c->d_stage_in, stride * c->P);
+        if (e == cudaSuccess) e = cudaMalloc(&c->d_stage_out, stride);
+        if (e != cudaSuccess) {
+            if (c->d_stage_in) { cudaFree(c->d_stage_in); c->d_stage_in = nullptr; }
+            cudaGetLastError();
+            set_error("sifar_allreduce_host: staging allocation failed: %s", cudaGetErrorString(e));
+            return SIFAR_ERR_NOMEM;
+        }
+    }
+    cudaStream_t s = c->host_stream;
+    const size_t bytes = n * elem_size(c->dtype);
+    for (int r = 0; r < c->P; ++r) {
+        if (!host_rank_ptrs[r]) { set_error("sifar_allreduce_host: NULL rank pointer"); return SIFAR_ERR_INVALID; }
+        if (bytes) SIFAR_CUDA(cudaMemcpyAsync(c->d_stage_in + r * stride, host_rank_ptrs[r], bytes, cudaMemcpyHostToDevice, s));
+        if ((rc = sifar_pack(c, r, c->d_stage_in + r * stride, n, mode, s))) return rc;
+    }
+    if ((rc = sifar_allreduce(c, nullptr, c->d_stage_out, n, mode, s))) return rc;
+    if (bytes) SIFAR_CUDA(cudaMemcpyAsync(host_out, c->d_stage_out, bytes, cudaMemcpyDeviceToHost, s));
+    SIFAR_CUDA(cudaStreamSynchronize(s));
+    rc = *c->h_status;
+    if (rc) set_error("sifar_allreduce_host: device status %d", rc);
+    return rc;
+}

@@ -1,0 +1,118 @@
+/*
+ * Internal declarations shared by the translation units of libsifar.so:
+ * the device-resident protocol state, the host context, launch helpers.
+ */
+#ifndef SIFAR_INTERNAL_CUH
+#define SIFAR_INTERNAL_CUH
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "sifar.h"
+#include "sifar_device.cuh"
+
+namespace sifar {
+
+constexpr int kMaxRanks = SIFAR_MAX_RANKS;
+constexpr uint32_t kEpochLimit = 0xFFFFFFFEu;    /* last usable call number                  */
+
+/*
+ * Protocol state in device memory (one per context, zero-filled at creation).
+ * Words that different actors poll sit in different 128-byte lines.
+ */
+struct __align__(128) DevState {
+    /* line 0: call number and sticky status; read together by every kernel at entry */
+    uint32_t epoch;                  /* number of completed calls                               */
+    uint32_t status;                 /* 0, or a negative sifar_status_t stored as uint32         */
+    uint32_t pad0[30];
+    /* line 1: last-CTA detection of the reducer; retry marker */
+    uint32_t cta_arrive;
+    uint32_t retry_epoch;            /* call number of the last call that re-loaded a slot       */
+    uint32_t pad1[30];
+    /* lines 2-3: arrival flags, one 128-byte line per parity (top barrier) */
+    uint32_t arrive[2][32];
+    /* line 4: done flags (bottom barrier, BARRIER_ONESHOT) */
+    uint32_t done[32];
+    /* line 5: per-rank CTA counters of the pack kernels */
+    uint32_t pack_count[32];
+    /* line 6: statistics */
+    unsigned long long stats[16];
+};
+
+enum StatIndex { kStatCalls = 0, kStatCallsWithRetry = 1, kStatSlotReloads = 2, kStatFlagPolls = 3,
+                 kStatTimeouts = 4 };
+
+/* Record a failed wait: sticky status on the device and in the host-mapped word. */
+__device__ __forceinline__ void fail(DevState *st, volatile int *host_status, int code)
+{
+    if (atomicCAS(&st->status, 0u, (uint32_t)code) == 0u) {
+        atomicAdd(&st->stats[kStatTimeouts], 1ull);
+        *host_status = code;
+        __threadfence_system();
+    }
+}
+
+/* Element geometry */
+__host__ __device__ inline size_t elem_size(int dtype) { return dtype == SIFAR_BF16 ? 2 : 4; }
+__host__ __device__ inline size_t elems_per_slot(int dtype) { return dtype == SIFAR_BF16 ? 6 : 3; }
+__host__ __device__ inline size_t slots_for(int dtype, size_t n)
+{
+    size_t k = elems_per_slot(dtype);
+    return (n + k - 1) / k;
+}
+
+}  /* namespace sifar */
+
+/* Host context. */
+struct sifar_ctx {
+    int P;
+    int dtype;
+    int device;
+    int sm_count;
+    size_t max_elems;
+    size_t plain_stride;             /* bytes between two rank buffers (multiple of 256) */
+    size_t slot_stride;
+    char *d_plain;                   /* [parity][rank] plain buffers                     */
+    char *d_slots;                   /* [parity][rank] slot buffers                      */
+    sifar::DevState *d_state;
+    volatile int *h_status;          /* pinned, mapped                                   */
+    int *d_status_alias;             /* device alias of h_status                         */
+    uint32_t h_epoch;                /* calls enqueued so far                            */
+    uint32_t last_mode0_epoch;       /* last BARRIER_ONESHOT call (0: none): whose done flags a producer waits for */
+    unsigned long long timeout_ns;
+    /* staging for sifar_allreduce_host, allocated on first use */
+    char *d_stage_in;
+    char *d_stage_out;
+    cudaStream_t host_stream;
+
+    char *plain_buf(int parity, int r) const { return d_plain + ((size_t)parity * P + r) * plain_stride; }
+    char *slot_buf(int parity, int r) const { return d_slots + ((size_t)parity * P + r) * slot_stride; }
+};
+
+namespace sifar {
+
+/* Error text of the calling thread. */
+void set_error(const char *fmt, ...);
+int cuda_fail(cudaError_t e, const char *what);
+
+#define SIFAR_CUDA(call)                                                   \
+    do {                                                                   \
+        cudaError_t e__ = (call);                                          \
+        if (e__ != cudaSuccess) return ::sifar::cuda_fail(e__, #call);     \
+    } while (0)
+
+/* Internal launchers, implemented in sifar_core.cu, used by the chains too. */
+struct ReduceLaunch {
+    const void *src[kMaxRanks];      /* parity-resolved rank buffers (plain or slots)   */
+    void *out;
+    size_t n;
+    int mode;
+    uint32_t parity;                 /* parity the host expects the call number to have */
+    int use_flags;                   /* barrier modes: poll arrival flags               */
+};
+
+int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream);
+
+}  /* namespace sifar */
+#endif
