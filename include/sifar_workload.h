@@ -1,0 +1,133 @@
+/*
+ * sifar_workload.h - synthetic decode-step workloads that drive the all-reduce:
+ * the chain of dependent {P producers -> all-reduce} steps of one token.
+ *
+ * The paper's setting (Sections 2.3, 3.5, 6.1): a decode step issues two
+ * all-reduces per transformer layer, each fed by an operation on the previous
+ * result, all inside one CUDA graph or one fused "megakernel" with no host
+ * involvement, and all-reduce latency is measured back to back inside that
+ * kernel.  Model weights are not available here, so "the next operation" of rank
+ * r is a seeded elementwise update of the previous result (rules below); what is
+ * kept is the dependency structure and the per-call traffic.
+ *
+ * Step t = 1, 2, ... of a chain (t = call number - call number at creation):
+ *   every rank r produces its partial x_r^t   (t = 1: from the generator;
+ *                                              t > 1: from out^{t-1});
+ *   out^t = all-reduce(x_0^t .. x_{P-1}^t)  in the chain's mode.
+ * Producers of step t are ordered after the all-reduce of step t-1 (they consume
+ * its result: stream event, graph edge, or a ready flag inside the persistent
+ * kernel) and are NOT ordered before the all-reduce of step t by anything but
+ * the arrival flags / slot tags of the mode under test.
+ *
+ * Update rules (each product and the sum rounded separately, no fused
+ * multiply-add; z = noise of (seed, rank, step, element)):
+ *   kind 0 (gauss, z ~ N(0,1) as a sum of twelve 16-bit uniforms) and
+ *   kind 2 (uniform, z ~ U[-1,1)):
+ *       x_r^1[i]   = narrow( z * (outlier(r,i) ? 100 : 1) )
+ *       x_r^t[i]   = narrow( widen(out^{t-1}[i]) * scale + z * sigma )
+ *   kind 1 (integers in [-64,64], k uniform on 0..128):
+ *       x_r^1[i]   = k - 64
+ *       x_r^t[i]   = ((int(out^{t-1}[i]) + k) mod 129, taken in [0,128]) - 64
+ * delay_max_ns > 0: before storing, rank r at step t busy-waits a seeded time
+ * uniform on [0, delay_max_ns] (skewed arrival); values are unaffected.
+ */
+#ifndef SIFAR_WORKLOAD_H
+#define SIFAR_WORKLOAD_H
+
+#include "sifar.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct {
+    int      kind;            /* 0 gauss, 1 integers, 2 uniform */
+    unsigned seed;
+    float    scale;
+    float    sigma;
+    unsigned outlier_mod;     /* 0: none; m: one first partial in m is multiplied by 100 */
+    unsigned delay_max_ns;
+} sifar_workload;
+
+typedef struct sifar_chain sifar_chain;   /* opaque */
+
+/* How the chain runs on the device. */
+typedef enum {
+    SIFAR_CHAIN_STREAMS    = 0,  /* P producer streams + one reducer stream, events for the result dependency   */
+    SIFAR_CHAIN_GRAPH      = 1,  /* the same topology captured once into a CUDA graph and replayed              */
+    SIFAR_CHAIN_PERSISTENT = 2   /* one cooperative kernel: reducer CTAs and P groups of producer CTAs that talk
+                                    only through flags / tags in memory, for all steps of a run                 */
+} sifar_chain_impl;
+
+/* Fourth "mode", chains only: no all-reduce at all; each rank's next operation consumes its own
+   partial (the paper's "feed the input of the all-reduce to the next operation" experiment, Section 2.3).
+   A timing floor; its results are not a sum. */
+enum { SIFAR_CHAIN_NO_ALLREDUCE = 3 };
+
+/* Bytes between two rows of an output ring for n elements (a multiple of 256). */
+size_t sifar_chain_ring_stride(int dtype, size_t n);
+
+/*
+ * Create a chain on `ctx` (which it then owns exclusively until destroyed: no other
+ * sifar_allreduce / sifar_pack on that context in between).
+ *   n              elements per rank, 1 <= n <= max_elems of the context
+ *   mode           a sifar_mode, or SIFAR_CHAIN_NO_ALLREDUCE
+ *   impl           a sifar_chain_impl
+ *   out_ring       device, ring_len rows of sifar_chain_ring_stride() bytes, caller-owned;
+ *                  out^t lands in row (t-1) mod ring_len (bytes of a row past n elements
+ *                  are unspecified)
+ *   ring_len       >= 2 and a divisor of steps_per_run
+ *   steps_per_run  even, >= 2
+ * Returns NULL on failure (sifar_last_error()).
+ */
+sifar_chain *sifar_chain_create(sifar_ctx *ctx, const sifar_workload *w, size_t n, int mode, int impl,
+                                void *out_ring, int ring_len, int steps_per_run);
+
+/* Enqueue the next steps_per_run steps on `stream`; consecutive runs continue the same chain. */
+int sifar_chain_run(sifar_chain *chain, void *stream);
+
+/*
+ * Device timestamps (nanoseconds, %globaltimer) of the last run, after it has
+ * finished: stamps[0] = start of the run, stamps[s] = result of step s of the run
+ * published, s = 1..steps_per_run.  PERSISTENT only (else SIFAR_ERR_INVALID).
+ * Synchronizes the device.
+ */
+int sifar_chain_stamps(sifar_chain *chain, unsigned long long *stamps);
+
+/* Kernels launched per run by this chain (graph replays count their kernel nodes). */
+int sifar_chain_launches_per_run(sifar_chain *chain);
+
+int sifar_chain_destroy(sifar_chain *chain);
+
+/*
+ * Generator probes (for tests and for building inputs on the device): write the
+ * first partial of `rank`, or its partial of step t >= 2 from prev_out, as n plain
+ * elements of `dtype` to dst (device, 16-byte aligned).
+ */
+int sifar_workload_first(const sifar_workload *w, int rank, int dtype, void *dst, size_t n, void *stream);
+int sifar_workload_next(const sifar_workload *w, int rank, unsigned t, int dtype, const void *prev_out,
+                        void *dst, size_t n, void *stream);
+/* The seeded producer delays of ranks 0..P-1 at step t, computed on the device, copied to host_out[P]. Synchronizes. */
+int sifar_workload_delays(const sifar_workload *w, int P, unsigned t, unsigned *host_out);
+
+/*
+ * Enqueue a kernel that busy-waits `ns` nanoseconds (at most 50 ms) on `stream`:
+ * used to force producer / reducer orderings in tests and benchmarks.
+ */
+int sifar_spin(unsigned ns, void *stream);
+
+/*
+ * 16-byte access atomicity check (the speculative slots rely on it): `writers`
+ * CTAs keep overwriting `nslots` slots with patterns whose four words all derive
+ * from one counter, while reader CTAs load them with the slot load and count
+ * slots whose words disagree.  Runs `rounds` rounds, all co-resident (cooperative
+ * launch), bounded.  *host_torn receives the number of torn observations,
+ * *host_reads the number of slot reads.  Synchronizes.
+ */
+int sifar_tear_check(unsigned nslots, unsigned rounds, unsigned long long *host_torn,
+                     unsigned long long *host_reads);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SIFAR_WORKLOAD_H */

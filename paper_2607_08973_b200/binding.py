@@ -142,3 +142,106 @@ def sifar_slot_count(dtype: int, n: int) -> int:
 
 def sifar_algorithmic_bytes(P: int, dtype: int, n: int, mode: int) -> int:
     return lib().sifar_algorithmic_bytes(P, dtype, n, mode)
+
+
+# ---------------------------------------------------------------------------
+# include/sifar_workload.h: synthetic decode-step chains
+# ---------------------------------------------------------------------------
+CHAIN_STREAMS, CHAIN_GRAPH, CHAIN_PERSISTENT = 0, 1, 2
+CHAIN_NO_ALLREDUCE = 3
+IMPL_NAMES = {CHAIN_STREAMS: "streams", CHAIN_GRAPH: "graph", CHAIN_PERSISTENT: "persistent"}
+
+
+class sifar_workload(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int), ("seed", ctypes.c_uint), ("scale", ctypes.c_float),
+                ("sigma", ctypes.c_float), ("outlier_mod", ctypes.c_uint), ("delay_max_ns", ctypes.c_uint)]
+
+
+def make_workload(kind: int, seed: int, scale: float, sigma: float, outlier_mod: int = 0,
+                  delay_max_ns: int = 0) -> sifar_workload:
+    return sifar_workload(kind, seed, scale, sigma, outlier_mod, delay_max_ns)
+
+
+_wl_ready = False
+
+
+def _wl() -> ctypes.CDLL:
+    global _wl_ready
+    L = lib()
+    if not _wl_ready:
+        vp, sz, ci, cu = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint
+        wp = ctypes.POINTER(sifar_workload)
+        ullp = ctypes.POINTER(ctypes.c_ulonglong)
+        sig = {
+            "sifar_chain_ring_stride": (sz, [ci, sz]),
+            "sifar_chain_create": (vp, [vp, wp, sz, ci, ci, vp, ci, ci]),
+            "sifar_chain_run": (ci, [vp, vp]),
+            "sifar_chain_stamps": (ci, [vp, ullp]),
+            "sifar_chain_launches_per_run": (ci, [vp]),
+            "sifar_chain_destroy": (ci, [vp]),
+            "sifar_workload_first": (ci, [wp, ci, ci, vp, sz, vp]),
+            "sifar_workload_next": (ci, [wp, ci, cu, ci, vp, vp, sz, vp]),
+            "sifar_workload_delays": (ci, [wp, ci, cu, ctypes.POINTER(cu)]),
+            "sifar_spin": (ci, [cu, vp]),
+            "sifar_tear_check": (ci, [cu, cu, ullp, ullp]),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _wl_ready = True
+    return L
+
+
+def sifar_chain_ring_stride(dtype: int, n: int) -> int:
+    return _wl().sifar_chain_ring_stride(dtype, n)
+
+
+def sifar_chain_create(ctx: int, w: sifar_workload, n: int, mode: int, impl: int, out_ring: int, ring_len: int,
+                       steps_per_run: int) -> int:
+    h = _wl().sifar_chain_create(ctx, ctypes.byref(w), n, mode, impl, out_ring, ring_len, steps_per_run)
+    if not h:
+        raise SifarError(ERR_INVALID, sifar_last_error())
+    return h
+
+
+def sifar_chain_run(chain: int, stream: int = 0) -> int:
+    return _check(_wl().sifar_chain_run(chain, stream))
+
+
+def sifar_chain_stamps(chain: int, steps_per_run: int) -> list[int]:
+    buf = (ctypes.c_ulonglong * (steps_per_run + 1))()
+    _check(_wl().sifar_chain_stamps(chain, buf))
+    return list(buf)
+
+
+def sifar_chain_launches_per_run(chain: int) -> int:
+    return _wl().sifar_chain_launches_per_run(chain)
+
+
+def sifar_chain_destroy(chain: int) -> int:
+    return _check(_wl().sifar_chain_destroy(chain))
+
+
+def sifar_workload_first(w: sifar_workload, rank: int, dtype: int, dst: int, n: int, stream: int = 0) -> int:
+    return _check(_wl().sifar_workload_first(ctypes.byref(w), rank, dtype, dst, n, stream))
+
+
+def sifar_workload_next(w: sifar_workload, rank: int, t: int, dtype: int, prev_out: int, dst: int, n: int,
+                        stream: int = 0) -> int:
+    return _check(_wl().sifar_workload_next(ctypes.byref(w), rank, t, dtype, prev_out, dst, n, stream))
+
+
+def sifar_workload_delays(w: sifar_workload, P: int, t: int) -> list[int]:
+    buf = (ctypes.c_uint * P)()
+    _check(_wl().sifar_workload_delays(ctypes.byref(w), P, t, buf))
+    return list(buf)
+
+
+def sifar_spin(ns: int, stream: int = 0) -> int:
+    return _check(_wl().sifar_spin(ns, stream))
+
+
+def sifar_tear_check(nslots: int, rounds: int) -> tuple[int, int]:
+    torn, reads = ctypes.c_ulonglong(), ctypes.c_ulonglong()
+    _check(_wl().sifar_tear_check(nslots, rounds, ctypes.byref(torn), ctypes.byref(reads)))
+    return torn.value, reads.value

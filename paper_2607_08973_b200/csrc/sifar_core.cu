@@ -28,6 +28,7 @@
 #include <new>
 
 #include "sifar_internal.cuh"
+#include "sifar_reduce.cuh"
 
 namespace sifar {
 
@@ -79,36 +80,8 @@ struct PackArgs {
 constexpr int kThreads = 256;
 
 /* ------------------------------------------------------------------------ */
-/* entry / exit of a reducer CTA                                             */
+/* exit of a reducer CTA                                                     */
 /* ------------------------------------------------------------------------ */
-
-/* Bounded poll of a flag until it equals `want` (acquire).  Returns the number of failed polls, or -1 on time-out. */
-__device__ __forceinline__ int wait_flag_eq(const uint32_t *flag, uint32_t want, unsigned long long timeout_ns)
-{
-    int polls = 0;
-    unsigned long long t0 = 0;
-    while (ld_acquire_u32(flag) != want) {
-        ++polls;
-        unsigned long long now = globaltimer_ns();
-        if (t0 == 0) t0 = now;
-        else if (now - t0 > timeout_ns) return -1;
-    }
-    return polls;
-}
-
-/* Same for "flag - base is in [0, 2^31)", i.e. flag has reached `base` (call numbers never wrap inside a context's life). */
-__device__ __forceinline__ int wait_flag_ge(const uint32_t *flag, uint32_t base, unsigned long long timeout_ns)
-{
-    int polls = 0;
-    unsigned long long t0 = 0;
-    while (ld_acquire_u32(flag) < base) {
-        ++polls;
-        unsigned long long now = globaltimer_ns();
-        if (t0 == 0) t0 = now;
-        else if (now - t0 > timeout_ns) return -1;
-    }
-    return polls;
-}
 
 /*
  * Completion of a reducer CTA, called by thread 0 after a __syncthreads().  The
@@ -130,45 +103,6 @@ __device__ __forceinline__ void reducer_finish(DevState *st, uint32_t e, int P)
         st_release_u32(&st->epoch, e);
     }
 }
-
-/* ------------------------------------------------------------------------ */
-/* rank-order accumulation                                                   */
-/* ------------------------------------------------------------------------ */
-template <int DT, int P>
-__device__ __forceinline__ uint32_t sum_word(const uint32_t (&w)[P])
-{
-    if (DT == SIFAR_BF16) {
-        float lo = bf16lo_to_f32(w[0]), hi = bf16hi_to_f32(w[0]);
-#pragma unroll
-        for (int r = 1; r < P; ++r) {
-            lo = __fadd_rn(lo, bf16lo_to_f32(w[r]));
-            hi = __fadd_rn(hi, bf16hi_to_f32(w[r]));
-        }
-        return f32x2_to_bf16x2(lo, hi);
-    } else {
-        float acc = __uint_as_float(w[0]);
-#pragma unroll
-        for (int r = 1; r < P; ++r) acc = __fadd_rn(acc, __uint_as_float(w[r]));
-        return __float_as_uint(acc);
-    }
-}
-
-template <int DT, int P>
-__device__ __forceinline__ uint4 sum_vec(const uint4 (&x)[P], bool with_w)
-{
-    uint32_t a[P], b[P], c[P], d[P];
-#pragma unroll
-    for (int r = 0; r < P; ++r) { a[r] = x[r].x; b[r] = x[r].y; c[r] = x[r].z; d[r] = x[r].w; }
-    uint4 o;
-    o.x = sum_word<DT, P>(a);
-    o.y = sum_word<DT, P>(b);
-    o.z = sum_word<DT, P>(c);
-    o.w = with_w ? sum_word<DT, P>(d) : 0u;
-    return o;
-}
-
-/* Vectors (plain) or slots (speculative) a thread keeps in flight per rank. */
-template <int P> struct Unroll { static constexpr int value = (P <= 2) ? 4 : (P <= 4) ? 2 : 1; };
 
 /* ------------------------------------------------------------------------ */
 /* reducer, barrier modes: plain partials behind arrival flags               */
@@ -291,49 +225,12 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
         for (int u = 0; u < U; ++u) {
             const size_t s = base + (size_t)u * kThreads;
             if (s >= nslots) continue;
-            /* Validation (Section 4.2): a slot counts iff it carries this call's tag. */
-            uint32_t stale = 0;
-#pragma unroll
-            for (int r = 0; r < P; ++r) stale |= (uint32_t)(x[u][r].w != e) << r;
-            if (stale) {
-                /* Mis-speculation: re-load only the stale ranks of this slot, with back-off, until the time limit. */
-                const unsigned long long t0 = globaltimer_ns();
-                unsigned spins = 0;
-                do {
-#pragma unroll
-                    for (int r = 0; r < P; ++r) {
-                        if (stale & (1u << r)) {
-                            x[u][r] = ld_slot(a.src[r] + s);
-                            ++reloads;
-                            if (x[u][r].w == e) stale &= ~(1u << r);
-                        }
-                    }
-                    if (stale) {
-                        if (globaltimer_ns() - t0 > a.timeout_ns) {
-                            fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
-                            alive = false;
-                            break;
-                        }
-                        if (++spins > 8) __nanosleep(spins > 64 ? 200 : 40);
-                    }
-                } while (stale);
-                if (!alive) break;
+            if (!validate_slot<P>(x[u], a.src, s, e, a.timeout_ns, reloads)) {
+                fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+                alive = false;
+                break;
             }
-            const uint4 o = sum_vec<DT, P>(x[u], false);
-            const size_t i0 = s * EPS;
-            if (i0 + EPS <= a.n) {
-                uint32_t *dst = reinterpret_cast<uint32_t *>(a.out) + s * 3;
-                dst[0] = o.x; dst[1] = o.y; dst[2] = o.z;
-            } else if (DT == SIFAR_BF16) {
-                uint16_t *dst = reinterpret_cast<uint16_t *>(a.out) + i0;
-                const uint32_t w[3] = {o.x, o.y, o.z};
-                for (int k = 0; k < EPS && i0 + k < a.n; ++k)
-                    dst[k] = (uint16_t)((w[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu);
-            } else {
-                uint32_t *dst = reinterpret_cast<uint32_t *>(a.out) + i0;
-                const uint32_t w[3] = {o.x, o.y, o.z};
-                for (int k = 0; k < EPS && i0 + k < a.n; ++k) dst[k] = w[k];
-            }
+            store_slot_result<DT>(a.out, s, (size_t)a.n, sum_vec<DT, P>(x[u], false));
         }
     }
 

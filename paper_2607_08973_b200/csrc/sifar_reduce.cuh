@@ -1,0 +1,166 @@
+/*
+ * Device-side pieces shared by the discrete reducer kernels and by the
+ * persistent decode-step chain: bounded flag waits, rank-order accumulation,
+ * slot validation with retry, masked result stores.
+ */
+#ifndef SIFAR_REDUCE_CUH
+#define SIFAR_REDUCE_CUH
+
+#include "sifar_internal.cuh"
+
+namespace sifar {
+
+/* ------------------------------------------------------------------------ */
+/* bounded waits                                                             */
+/* ------------------------------------------------------------------------ */
+
+/* Bounded poll of a flag until it equals `want` (acquire).  Returns the number of failed polls, or -1 on time-out. */
+__device__ __forceinline__ int wait_flag_eq(const uint32_t *flag, uint32_t want, unsigned long long timeout_ns)
+{
+    int polls = 0;
+    unsigned long long t0 = 0;
+    while (ld_acquire_u32(flag) != want) {
+        ++polls;
+        unsigned long long now = globaltimer_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > timeout_ns) return -1;
+    }
+    return polls;
+}
+
+/* Same for "flag - base is in [0, 2^31)", i.e. flag has reached `base` (call numbers never wrap inside a context's life). */
+__device__ __forceinline__ int wait_flag_ge(const uint32_t *flag, uint32_t base, unsigned long long timeout_ns)
+{
+    int polls = 0;
+    unsigned long long t0 = 0;
+    while (ld_acquire_u32(flag) < base) {
+        ++polls;
+        unsigned long long now = globaltimer_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > timeout_ns) return -1;
+    }
+    return polls;
+}
+
+/* ------------------------------------------------------------------------ */
+/* rank-order accumulation                                                   */
+/* ------------------------------------------------------------------------ */
+template <int DT, int P>
+__device__ __forceinline__ uint32_t sum_word(const uint32_t (&w)[P])
+{
+    if (DT == SIFAR_BF16) {
+        float lo = bf16lo_to_f32(w[0]), hi = bf16hi_to_f32(w[0]);
+#pragma unroll
+        for (int r = 1; r < P; ++r) {
+            lo = __fadd_rn(lo, bf16lo_to_f32(w[r]));
+            hi = __fadd_rn(hi, bf16hi_to_f32(w[r]));
+        }
+        return f32x2_to_bf16x2(lo, hi);
+    } else {
+        float acc = __uint_as_float(w[0]);
+#pragma unroll
+        for (int r = 1; r < P; ++r) acc = __fadd_rn(acc, __uint_as_float(w[r]));
+        return __float_as_uint(acc);
+    }
+}
+
+template <int DT, int P>
+__device__ __forceinline__ uint4 sum_vec(const uint4 (&x)[P], bool with_w)
+{
+    uint32_t a[P], b[P], c[P], d[P];
+#pragma unroll
+    for (int r = 0; r < P; ++r) { a[r] = x[r].x; b[r] = x[r].y; c[r] = x[r].z; d[r] = x[r].w; }
+    uint4 o;
+    o.x = sum_word<DT, P>(a);
+    o.y = sum_word<DT, P>(b);
+    o.z = sum_word<DT, P>(c);
+    o.w = with_w ? sum_word<DT, P>(d) : 0u;
+    return o;
+}
+
+/* Vectors (plain) or slots (speculative) a thread keeps in flight per rank. */
+template <int P> struct Unroll { static constexpr int value = (P <= 2) ? 4 : (P <= 4) ? 2 : 1; };
+
+/* ------------------------------------------------------------------------ */
+/* slot validation (speculative mode)                                        */
+/* ------------------------------------------------------------------------ */
+/*
+ * x[r] holds rank r's slot `s` as first loaded.  A slot counts iff its tag equals
+ * the call number e (Section 4.2: validation after the speculative read).  On
+ * mis-speculation only the stale ranks of this slot are loaded again, with a
+ * short back-off, until every tag matches or the time limit passes.  Returns
+ * false on time-out.  `reloads` counts the extra loads.
+ */
+template <int P>
+__device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const *src, size_t s, uint32_t e,
+                                              unsigned long long timeout_ns, unsigned &reloads)
+{
+    uint32_t stale = 0;
+#pragma unroll
+    for (int r = 0; r < P; ++r) stale |= (uint32_t)(x[r].w != e) << r;
+    if (stale == 0u) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    unsigned spins = 0;
+    do {
+#pragma unroll
+        for (int r = 0; r < P; ++r) {
+            if (stale & (1u << r)) {
+                x[r] = ld_slot(src[r] + s);
+                ++reloads;
+                if (x[r].w == e) stale &= ~(1u << r);
+            }
+        }
+        if (stale) {
+            if (globaltimer_ns() - t0 > timeout_ns) return false;
+            if (++spins > 8) __nanosleep(spins > 64 ? 200 : 40);
+        }
+    } while (stale);
+    return true;
+}
+
+/* ------------------------------------------------------------------------ */
+/* result stores                                                             */
+/* ------------------------------------------------------------------------ */
+/* The 12 data bytes of reduced slot s go to elements [s*EPS, s*EPS+EPS) of out; a short last slot is masked. */
+template <int DT>
+__device__ __forceinline__ void store_slot_result(void *out, size_t s, size_t n, const uint4 &o)
+{
+    constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;
+    const size_t i0 = s * EPS;
+    if (i0 + EPS <= n) {
+        uint32_t *dst = reinterpret_cast<uint32_t *>(out) + s * 3;
+        dst[0] = o.x; dst[1] = o.y; dst[2] = o.z;
+    } else if (DT == SIFAR_BF16) {
+        uint16_t *dst = reinterpret_cast<uint16_t *>(out) + i0;
+        const uint32_t w[3] = {o.x, o.y, o.z};
+        for (int k = 0; k < EPS && i0 + k < n; ++k)
+            dst[k] = (uint16_t)((w[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu);
+    } else {
+        uint32_t *dst = reinterpret_cast<uint32_t *>(out) + i0;
+        const uint32_t w[3] = {o.x, o.y, o.z};
+        for (int k = 0; k < EPS && i0 + k < n; ++k) dst[k] = w[k];
+    }
+}
+
+/* Reduced 16-byte vector v goes to elements [v*EPV, v*EPV+EPV) of out; a short last vector is masked. */
+template <int DT>
+__device__ __forceinline__ void store_vec_result(void *out, size_t v, size_t n, const uint4 &o)
+{
+    constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
+    const size_t i0 = v * EPV;
+    if (i0 + EPV <= n) {
+        reinterpret_cast<uint4 *>(out)[v] = o;
+    } else if (DT == SIFAR_BF16) {
+        uint16_t *dst = reinterpret_cast<uint16_t *>(out) + i0;
+        const uint32_t w[4] = {o.x, o.y, o.z, o.w};
+        for (int k = 0; k < EPV && i0 + k < n; ++k)
+            dst[k] = (uint16_t)((w[k >> 1] >> ((k & 1) * 16)) & 0xFFFFu);
+    } else {
+        uint32_t *dst = reinterpret_cast<uint32_t *>(out) + i0;
+        const uint32_t w[4] = {o.x, o.y, o.z, o.w};
+        for (int k = 0; k < EPV && i0 + k < n; ++k) dst[k] = w[k];
+    }
+}
+
+}  /* namespace sifar */
+#endif

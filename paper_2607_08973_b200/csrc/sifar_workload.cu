@@ -1,0 +1,945 @@
+/*
+ * sifar_workload.cu - synthetic decode-step chains around the all-reduce:
+ * seeded producer kernels, and the three ways a chain of dependent
+ * {P producers -> all-reduce} steps runs on the device (streams + events, one
+ * CUDA graph, one cooperative persistent kernel).
+ *
+ * The persistent kernel is the analogue of measuring all-reduces back to back
+ * inside a fused forward-pass kernel (paper, Sections 4.2 "Megakernel
+ * Integration" and 6.1): no launch or graph-edge latency separates the steps, so
+ * what differs between the modes is exactly the synchronization they perform:
+ *
+ *   BARRIER_ONESHOT : ready -> [done wait] produce -> arrival flag -> flag poll
+ *                     -> load/sum/store -> ready; all reducer CTAs arrive, done flags
+ *   DUALBUF         : ready -> produce -> arrival flag -> flag poll -> load/sum/store -> ready
+ *   SPECULATIVE     : ready -> produce tagged slots -> load/validate/sum/store -> ready
+ *
+ * where "ready" is the result-ready flag that models ordinary same-GPU operator
+ * ordering (identical in all modes) and every arrow is one dependent trip
+ * through the L2.
+ */
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "sifar_internal.cuh"
+#include "sifar_reduce.cuh"
+#include "sifar_workload.h"
+
+namespace sifar {
+
+/* ------------------------------------------------------------------------ */
+/* counter generator (device restatement; integer-only, exact in binary32)   */
+/* ------------------------------------------------------------------------ */
+__host__ __device__ __forceinline__ uint32_t mix32(uint32_t x)
+{
+    x ^= x >> 16; x *= 0x7FEB352Du;
+    x ^= x >> 15; x *= 0x846CA68Bu;
+    x ^= x >> 16;
+    return x;
+}
+
+enum { kStreamValue = 1, kStreamOutlier = 2, kStreamDelay = 3 };
+
+/* The first four of the six chained mixes depend only on (seed, stream, rank, step). */
+__host__ __device__ __forceinline__ uint32_t gen_prefix(uint32_t seed, uint32_t stream, uint32_t r, uint32_t t)
+{
+    uint32_t h = mix32(seed);
+    h = mix32(h ^ stream);
+    h = mix32(h + r);
+    return mix32(h ^ (t * 0x9E3779B9u));
+}
+
+__host__ __device__ __forceinline__ uint32_t gen_word(uint32_t prefix, uint32_t i, uint32_t k)
+{
+    return mix32(mix32(prefix + i) ^ k);
+}
+
+struct Gen {
+    uint32_t value_prefix;     /* (seed, value stream, rank, step)   */
+    uint32_t outlier_prefix;   /* (seed, outlier stream, rank, 0)    */
+    int kind;
+    float scale, sigma;
+    uint32_t outlier_mod;
+};
+
+__device__ __forceinline__ Gen make_gen(const sifar_workload &w, uint32_t r, uint32_t t)
+{
+    Gen g;
+    g.value_prefix = gen_prefix(w.seed, kStreamValue, r, t);
+    g.outlier_prefix = gen_prefix(w.seed, kStreamOutlier, r, 0u);
+    g.kind = w.kind; g.scale = w.scale; g.sigma = w.sigma; g.outlier_mod = w.outlier_mod;
+    return g;
+}
+
+__device__ __forceinline__ float gen_uniform(const Gen &g, uint32_t i)
+{
+    const int32_t c = (int32_t)(gen_word(g.value_prefix, i, 0u) >> 8) - (1 << 23);
+    return __fmul_rn((float)c, 1.0f / 8388608.0f);
+}
+
+__device__ __forceinline__ float gen_gauss(const Gen &g, uint32_t i)
+{
+    int32_t s = 0;
+#pragma unroll
+    for (uint32_t k = 0; k < 6; ++k) {
+        const uint32_t w = gen_word(g.value_prefix, i, k);
+        s += (int32_t)(w & 0xFFFFu) + (int32_t)(w >> 16);
+    }
+    return __fmul_rn((float)(s - 393210), 1.0f / 65536.0f);
+}
+
+__device__ __forceinline__ int32_t gen_int129(const Gen &g, uint32_t i)
+{
+    return (int32_t)(gen_word(g.value_prefix, i, 0u) % 129u);
+}
+
+__device__ __forceinline__ uint32_t gen_delay_ns(const sifar_workload &w, uint32_t r, uint32_t t)
+{
+    if (w.delay_max_ns == 0u) return 0u;
+    return gen_word(gen_prefix(w.seed, kStreamDelay, r, t), 0u, 0u) % (w.delay_max_ns + 1u);
+}
+
+__device__ __forceinline__ float first_value(const Gen &g, uint32_t i)
+{
+    if (g.kind == 1) return (float)(gen_int129(g, i) - 64);
+    float z = (g.kind == 2) ? gen_uniform(g, i) : gen_gauss(g, i);
+    if (g.outlier_mod != 0u && gen_word(g.outlier_prefix, i, 0u) % g.outlier_mod == 0u) z = __fmul_rn(z, 100.0f);
+    return z;
+}
+
+__device__ __forceinline__ float next_value(const Gen &g, uint32_t i, float prev)
+{
+    if (g.kind == 1) {
+        int32_t v = ((int32_t)prev + gen_int129(g, i)) % 129;
+        if (v < 0) v += 129;
+        return (float)(v - 64);
+    }
+    const float z = (g.kind == 2) ? gen_uniform(g, i) : gen_gauss(g, i);
+    return __fadd_rn(__fmul_rn(prev, g.scale), __fmul_rn(z, g.sigma));
+}
+
+/*
+ * One unit of a rank's partial: NW 32-bit words starting at element i0 (bf16: two
+ * elements per word), elements at or past n are zero.  `prev` is out^{t-1}
+ * (ignored when `first`); it is read with strong loads because inside the
+ * persistent kernel it was written by another CTA of the same launch.
+ */
+template <int DT, int NW>
+__device__ __forceinline__ void produce_words(const Gen &g, bool first, const void *prev, size_t i0, size_t n,
+                                              uint32_t (&w)[NW])
+{
+    constexpr int EPW = (DT == SIFAR_BF16) ? 2 : 1;
+    uint32_t pw[NW];
+#pragma unroll
+    for (int j = 0; j < NW; ++j) pw[j] = 0u;
+    const bool full = (i0 + (size_t)NW * EPW <= n);
+    if (!first) {
+        if (full) {
+            const uint32_t *p32 = reinterpret_cast<const uint32_t *>(prev) + i0 / EPW;
+            if (NW == 4) {
+                const uint4 v = ld_slot(reinterpret_cast<const uint4 *>(p32));
+                pw[0] = v.x; pw[1] = v.y; pw[2] = v.z; pw[NW - 1] = v.w;
+            } else {
+#pragma unroll
+                for (int j = 0; j < NW; ++j) pw[j] = ld_relaxed_u32(p32 + j);
+            }
+        } else if (DT == SIFAR_BF16) {
+            const uint16_t *p16 = reinterpret_cast<const uint16_t *>(prev);
+            for (int k = 0; k < NW * 2 && i0 + k < n; ++k)
+                pw[k >> 1] |= (uint32_t)ld_relaxed_u16(p16 + i0 + k) << ((k & 1) * 16);
+        } else {
+            const uint32_t *p32 = reinterpret_cast<const uint32_t *>(prev);
+            for (int k = 0; k < NW && i0 + k < n; ++k) pw[k] = ld_relaxed_u32(p32 + i0 + k);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < NW; ++j) {
+        if (DT == SIFAR_BF16) {
+            const size_t ia = i0 + 2 * j, ib = ia + 1;
+            float a = 0.0f, b = 0.0f;
+            if (ia < n) a = first ? first_value(g, (uint32_t)ia) : next_value(g, (uint32_t)ia, bf16lo_to_f32(pw[j]));
+            if (ib < n) b = first ? first_value(g, (uint32_t)ib) : next_value(g, (uint32_t)ib, bf16hi_to_f32(pw[j]));
+            w[j] = f32x2_to_bf16x2(a, b);
+            if (ia >= n) w[j] = 0u;
+            else if (ib >= n) w[j] &= 0xFFFFu;
+        } else {
+            const size_t ia = i0 + j;
+            w[j] = 0u;
+            if (ia < n)
+                w[j] = __float_as_uint(first ? first_value(g, (uint32_t)ia)
+                                             : next_value(g, (uint32_t)ia, __uint_as_float(pw[j])));
+        }
+    }
+}
+
+/* Busy-wait `ns` nanoseconds on the global timer (ns is small and bounded by the caller). */
+__device__ __forceinline__ void spin_ns(uint32_t ns)
+{
+    if (ns == 0u) return;
+    const unsigned long long t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < (unsigned long long)ns) { }
+}
+
+constexpr int kModeNoAllreduce = SIFAR_CHAIN_NO_ALLREDUCE;
+constexpr unsigned kMaxDelayNs = 1000000u;       /* producer delays are capped at 1 ms */
+
+/* ------------------------------------------------------------------------ */
+/* producer kernel of the stream / graph chains                              */
+/* ------------------------------------------------------------------------ */
+struct ProduceArgs {
+    DevState *st;
+    int *host_status;
+    unsigned long long timeout_ns;
+    sifar_workload w;
+    uint32_t rank;
+    unsigned long long n;
+    const void *prev;          /* out^{t-1} (or the rank's own previous partial without all-reduce) */
+    void *dst;                 /* the rank's buffer of this step                                    */
+    uint32_t base_epoch;       /* step t = call number - base_epoch                                 */
+    uint32_t parity;
+    uint32_t t_fixed;          /* no-all-reduce chains: the step, since no call number advances     */
+};
+
+constexpr int kProdThreads = 128;
+
+template <int DT, int MODE>
+__global__ void __launch_bounds__(kProdThreads) k_produce(const ProduceArgs a)
+{
+    DevState *st = a.st;
+    __shared__ uint32_t s_e, s_t;
+    if (threadIdx.x == 0) {
+        uint32_t e = 0, t = a.t_fixed;
+        bool ok = true;
+        if (MODE != kModeNoAllreduce) {
+            const uint2 es = ld_relaxed_u32x2(&st->epoch);
+            e = es.x + 1u;
+            t = e - a.base_epoch;
+            ok = (es.y == 0u);
+            if (ok && MODE != SIFAR_BARRIER_ONESHOT && (e & 1u) != a.parity) {
+                fail(st, a.host_status, SIFAR_ERR_EPOCH);
+                ok = false;
+            }
+            /* bottom barrier, producer side: the single buffer may be overwritten once its last reader is done */
+            if (ok && MODE == SIFAR_BARRIER_ONESHOT && t > 1u &&
+                wait_flag_ge(&st->done[a.rank], e - 1u, a.timeout_ns) < 0) {
+                fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+                ok = false;
+            }
+        }
+        if (ok) spin_ns(gen_delay_ns(a.w, a.rank, t));
+        s_e = ok ? (MODE == kModeNoAllreduce ? 1u : e) : 0u;
+        s_t = t;
+    }
+    __syncthreads();
+    const uint32_t e = s_e, t = s_t;
+    if (e == 0u) return;
+
+    const Gen g = make_gen(a.w, a.rank, t);
+    const bool first = (t == 1u);
+    const size_t n = (size_t)a.n;
+    const size_t tid = (size_t)blockIdx.x * kProdThreads + threadIdx.x;
+    const size_t nthreads = (size_t)gridDim.x * kProdThreads;
+    if (MODE == SIFAR_SPECULATIVE) {
+        constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;
+        const size_t nslots = (n + EPS - 1) / EPS;
+        for (size_t s = tid; s < nslots; s += nthreads) {
+            uint32_t w[3];
+            produce_words<DT, 3>(g, first, a.prev, s * EPS, n, w);
+            store_slot(reinterpret_cast<uint4 *>(a.dst), s, w[0], w[1], w[2], e);
+        }
+    } else {
+        constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
+        const size_t nvec = (n + EPV - 1) / EPV;       /* the last vector is zero-padded inside the context's buffer */
+        for (size_t v = tid; v < nvec; v += nthreads) {
+            uint32_t w[4];
+            produce_words<DT, 4>(g, first, a.prev, v * EPV, n, w);
+            st_slot(reinterpret_cast<uint4 *>(a.dst) + v, make_uint4(w[0], w[1], w[2], w[3]));
+        }
+        if (MODE != kModeNoAllreduce)
+            signal_arrival(&st->pack_count[a.rank], gridDim.x, &st->arrive[e & 1u][a.rank], e);
+    }
+}
+
+/* Generator probes: plain elements to dst, no protocol. */
+template <int DT>
+__global__ void k_probe(sifar_workload w, uint32_t rank, uint32_t t, const void *prev, void *dst, unsigned long long n)
+{
+    constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
+    const Gen g = make_gen(w, rank, t);
+    const size_t nvec = ((size_t)n + EPV - 1) / EPV;
+    for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += (size_t)gridDim.x * blockDim.x) {
+        uint32_t wds[4];
+        produce_words<DT, 4>(g, t == 1u, prev, v * EPV, (size_t)n, wds);
+        store_vec_result<DT>(dst, v, (size_t)n, make_uint4(wds[0], wds[1], wds[2], wds[3]));
+    }
+}
+
+__global__ void k_delays(sifar_workload w, int P, uint32_t t, unsigned *out)
+{
+    if ((int)threadIdx.x < P) out[threadIdx.x] = gen_delay_ns(w, threadIdx.x, t);
+}
+
+__global__ void k_spin(unsigned ns) { spin_ns(ns); }
+
+/* ------------------------------------------------------------------------ */
+/* persistent chain kernel                                                   */
+/* ------------------------------------------------------------------------ */
+struct __align__(128) ChunkFlags {
+    uint32_t ready;                 /* call number whose result chunk is published                  */
+    uint32_t pad0[7];
+    uint32_t arrive[2][8];          /* per parity, per rank: this chunk of the rank's partial stored */
+    uint32_t pad1[8];
+};
+
+struct __align__(128) ChainDev {
+    uint32_t bottom_count;          /* reducer CTAs that finished reading (monotonic)               */
+    uint32_t exit_count;            /* CTAs that left the kernel (monotonic)                        */
+    uint32_t pad0[30];
+    uint32_t done[32];              /* bottom barrier, per rank                                     */
+};
+
+struct PersistArgs {
+    DevState *st;
+    int *host_status;
+    unsigned long long timeout_ns;
+    sifar_workload w;
+    unsigned long long n;
+    char *plain;                    /* [parity][rank] plain buffers */
+    unsigned long long plain_stride;
+    char *slots;                    /* [parity][rank] slot buffers  */
+    unsigned long long slot_stride;
+    char *ring;
+    unsigned long long ring_stride;
+    uint32_t ring_len;
+    uint32_t e0;                    /* calls completed before this run     */
+    uint32_t base_epoch;
+    uint32_t steps;
+    uint32_t C;                     /* chunks = reducer CTAs               */
+    uint32_t K;                     /* units per thread and step           */
+    uint32_t bottom_base, exit_base;
+    ChainDev *cs;
+    ChunkFlags *chunks;
+    unsigned long long *stamps;     /* steps + 1                           */
+    uint32_t *retry_steps;          /* steps: 1 if any CTA re-loaded a slot in that step */
+};
+
+constexpr int kChainThreads = 128;
+
+/* Bounded wait that also gives up when another CTA has already recorded a failure. */
+template <bool GE>
+__device__ __forceinline__ bool chain_wait(const uint32_t *flag, uint32_t want, DevState *st, int *host_status,
+                                           unsigned long long timeout_ns)
+{
+    unsigned long long t0 = 0;
+    unsigned polls = 0;
+    for (;;) {
+        const uint32_t v = ld_acquire_u32(flag);
+        if (GE ? (v >= want) : (v == want)) return true;
+        const unsigned long long now = globaltimer_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > timeout_ns) { fail(st, host_status, SIFAR_ERR_TIMEOUT); return false; }
+        if ((++polls & 63u) == 0u && ld_relaxed_u32(&st->status) != 0u) return false;
+    }
+}
+
+template <int DT, int P, int MODE>
+__global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
+{
+    DevState *st = a.st;
+    const uint32_t C = a.C;
+    const bool no_ar = (MODE == kModeNoAllreduce);
+    const bool is_reducer = !no_ar && blockIdx.x < C;
+    const uint32_t pidx = no_ar ? blockIdx.x : blockIdx.x - C;
+    const uint32_t rank = is_reducer ? 0u : pidx / C;
+    const uint32_t chunk = is_reducer ? blockIdx.x : pidx % C;
+    ChunkFlags *cf = a.chunks + chunk;
+    const size_t n = (size_t)a.n;
+    constexpr int EPU = (MODE == SIFAR_SPECULATIVE) ? ((DT == SIFAR_BF16) ? 6 : 3) : ((DT == SIFAR_BF16) ? 8 : 4);
+    const size_t nunits = (n + EPU - 1) / EPU;
+    const size_t unit0 = (size_t)chunk * kChainThreads * a.K + threadIdx.x;
+    __shared__ int s_ok;
+    unsigned reloads = 0;
+    bool alive = true;
+    const bool stamper = (blockIdx.x == 0);     /* reducer of chunk 0 (or rank 0's producer of chunk 0 without all-reduce) */
+    if (stamper && threadIdx.x == 0) a.stamps[0] = globaltimer_ns();
+
+    for (uint32_t s = 0; s < a.steps && alive; ++s) {
+        const uint32_t e = a.e0 + 1u + s;
+        const uint32_t t = e - a.base_epoch;
+        const uint32_t p = e & 1u;
+        char *ring_row = a.ring + (size_t)((t - 1u) % a.ring_len) * a.ring_stride;
+
+        if (is_reducer) {
+            /* ---------------- the pulling side ---------------- */
+            const uint4 *src[P];
+#pragma unroll
+            for (int r = 0; r < P; ++r) {
+                if (MODE == SIFAR_SPECULATIVE)
+                    src[r] = reinterpret_cast<const uint4 *>(a.slots + ((size_t)p * P + r) * a.slot_stride);
+                else
+                    src[r] = reinterpret_cast<const uint4 *>(
+                        a.plain + ((size_t)(MODE == SIFAR_DUALBUF ? p : 0u) * P + r) * a.plain_stride);
+            }
+            if (MODE != SIFAR_SPECULATIVE) {
+                /* top barrier: this chunk of every rank's partial has been stored */
+                if (threadIdx.x < 32) {
+                    bool ok = true;
+                    if (threadIdx.x < P)
+                        ok = chain_wait<false>(&cf->arrive[p][threadIdx.x], e, st, a.host_status, a.timeout_ns);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (threadIdx.x == 0) s_ok = ok;
+                }
+                __syncthreads();
+                if (!s_ok) { alive = false; break; }
+            }
+            bool retried = false;
+            for (uint32_t k = 0; k < a.K; ++k) {
+                const size_t u = unit0 + (size_t)k * kChainThreads;
+                if (u >= nunits) break;
+                uint4 x[P];
+#pragma unroll
+                for (int r = 0; r < P; ++r) x[r] = ld_slot(src[r] + u);
+                if (MODE == SIFAR_SPECULATIVE) {
+                    const unsigned before = reloads;
+                    if (!validate_slot<P>(x, src, u, e, a.timeout_ns, reloads)) {
+                        fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+                        alive = false;
+                        break;
+                    }
+                    retried |= (reloads != before);
+                    store_slot_result<DT>(ring_row, u, n, sum_vec<DT, P>(x, false));
+                } else {
+                    store_vec_result<DT>(ring_row, u, n, sum_vec<DT, P>(x, true));
+                }
+            }
+            if (MODE == SIFAR_SPECULATIVE && retried) st_relaxed_u32(&a.retry_steps[s], 1u);
+            if (!__syncthreads_and(alive)) { alive = false; break; }
+            if (threadIdx.x == 0) {
+                st_release_u32(&cf->ready, e);                 /* result chunk published */
+                if (stamper) a.stamps[s + 1u] = globaltimer_ns();
+                if (MODE == SIFAR_BARRIER_ONESHOT) {
+                    /* bottom barrier, reducer side: last CTA to finish reading releases the done flags */
+                    const uint32_t arrived = atom_add_acq_rel_u32(&a.cs->bottom_count, 1u) + 1u;
+                    if (arrived == a.bottom_base + (s + 1u) * C)
+                        for (int r = 0; r < P; ++r) st_release_u32(&a.cs->done[r], e);
+                }
+            }
+        } else {
+            /* ---------------- rank `rank`, chunk `chunk` of the next operation ---------------- */
+            if (threadIdx.x == 0) {
+                bool ok = true;
+                if (!no_ar && t > 1u) {
+                    ok = chain_wait<true>(&cf->ready, e - 1u, st, a.host_status, a.timeout_ns);
+                    if (ok && MODE == SIFAR_BARRIER_ONESHOT)
+                        ok = chain_wait<true>(&a.cs->done[rank], e - 1u, st, a.host_status, a.timeout_ns);
+                }
+                if (ok) spin_ns(gen_delay_ns(a.w, rank, t));
+                s_ok = ok;
+            }
+            __syncthreads();
+            if (!s_ok) { alive = false; break; }
+            const Gen g = make_gen(a.w, rank, t);
+            const bool first = (t == 1u);
+            const char *prev = no_ar ? a.plain + ((size_t)(p ^ 1u) * P + rank) * a.plain_stride
+                                     : a.ring + (size_t)((t + a.ring_len - 2u) % a.ring_len) * a.ring_stride;
+            for (uint32_t k = 0; k < a.K; ++k) {
+                const size_t u = unit0 + (size_t)k * kChainThreads;
+                if (u >= nunits) break;
+                if (MODE == SIFAR_SPECULATIVE) {
+                    uint32_t w[3];
+                    produce_words<DT, 3>(g, first, prev, u * EPU, n, w);
+                    store_slot(reinterpret_cast<uint4 *>(a.slots + ((size_t)p * P + rank) * a.slot_stride), u,
+                               w[0], w[1], w[2], e);
+                } else {
+                    uint32_t w[4];
+                    produce_words<DT, 4>(g, first, prev, u * EPU, n, w);
+                    const uint32_t bp = (MODE == SIFAR_BARRIER_ONESHOT) ? 0u : p;
+                    st_slot(reinterpret_cast<uint4 *>(a.plain + ((size_t)bp * P + rank) * a.plain_stride) + u,
+                            make_uint4(w[0], w[1], w[2], w[3]));
+                }
+            }
+            if (MODE == SIFAR_BARRIER_ONESHOT || MODE == SIFAR_DUALBUF) {
+                __syncthreads();
+                if (threadIdx.x == 0) st_release_u32(&cf->arrive[p][rank], e);
+            } else if (no_ar) {
+                __syncthreads();
+                if (stamper && threadIdx.x == 0) a.stamps[s + 1u] = globaltimer_ns();
+            }
+        }
+    }
+
+    /* leave: mis-speculation counters, then the last CTA out publishes the call number */
+    const unsigned warp_reloads = __reduce_add_sync(0xFFFFFFFFu, reloads);
+    if (warp_reloads && (threadIdx.x & 31) == 0)
+        atomicAdd(&st->stats[kStatSlotReloads], (unsigned long long)warp_reloads);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t left = atom_add_acq_rel_u32(&a.cs->exit_count, 1u) + 1u;
+        if (left == a.exit_base + gridDim.x && !no_ar && ld_relaxed_u32(&st->status) == 0u) {
+            unsigned long long with_retry = 0;
+            for (uint32_t s = 0; s < a.steps; ++s) {
+                with_retry += ld_relaxed_u32(&a.retry_steps[s]);
+                st_relaxed_u32(&a.retry_steps[s], 0u);
+            }
+            st->stats[kStatCalls] += a.steps;
+            st->stats[kStatCallsWithRetry] += with_retry;
+            st_release_u32(&st->epoch, a.e0 + a.steps);
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* 16-byte atomicity check                                                   */
+/* ------------------------------------------------------------------------ */
+__device__ __forceinline__ uint4 tear_pattern(uint32_t c)
+{
+    return make_uint4(c, ~c, c * 0x9E3779B9u, c ^ 0xA5A5A5A5u);
+}
+
+__global__ void __launch_bounds__(256) k_tear(uint4 *slots, unsigned nslots, unsigned rounds, unsigned writers,
+                                              unsigned long long *torn, unsigned long long *reads)
+{
+    const bool writer = blockIdx.x < writers;
+    unsigned long long my_torn = 0, my_reads = 0;
+    if (writer) {
+        const unsigned wid = blockIdx.x * blockDim.x + threadIdx.x, nw = writers * blockDim.x;
+        for (unsigned round = 1; round <= rounds; ++round)
+            for (unsigned s = wid; s < nslots; s += nw) st_slot(slots + s, tear_pattern(round * 2654435761u + s));
+    } else {
+        const unsigned rid = (blockIdx.x - writers) * blockDim.x + threadIdx.x;
+        const unsigned nr = (gridDim.x - writers) * blockDim.x;
+        for (unsigned round = 1; round <= rounds; ++round)
+            for (unsigned s = rid; s < nslots; s += nr) {
+                const uint4 v = ld_slot(slots + s);
+                const uint4 want = tear_pattern(v.x);
+                ++my_reads;
+                if (!(v.x == 0u && v.y == 0u && v.z == 0u && v.w == 0u) &&
+                    (v.y != want.y || v.z != want.z || v.w != want.w))
+                    ++my_torn;
+            }
+    }
+    if (my_torn) atomicAdd(torn, my_torn);
+    if (my_reads) atomicAdd(reads, my_reads);
+}
+
+}  /* namespace sifar */
+
+using namespace sifar;
+
+/* ------------------------------------------------------------------------ */
+/* host side                                                                 */
+/* ------------------------------------------------------------------------ */
+struct sifar_chain {
+    sifar_ctx *ctx;
+    sifar_workload w;
+    size_t n;
+    int mode, impl;
+    char *ring;
+    int ring_len;
+    size_t ring_stride;
+    int steps;
+    uint32_t base_epoch;
+    uint32_t runs;
+    int launches_per_run;
+    cudaStream_t prod[kMaxRanks];
+    cudaStream_t red;
+    cudaEvent_t ev_fork;
+    cudaEvent_t ev_join[kMaxRanks + 1];
+    std::vector<cudaEvent_t> ev_step;
+    cudaGraph_t graph;
+    cudaGraphExec_t exec;
+    /* persistent */
+    ChainDev *d_cs;
+    ChunkFlags *d_chunks;
+    unsigned long long *d_stamps;
+    uint32_t *d_retry_steps;
+    uint32_t C, K;
+    int grid;
+};
+
+static bool valid_workload(const sifar_workload *w)
+{
+    return w && w->kind >= 0 && w->kind <= 2 && w->delay_max_ns <= kMaxDelayNs;
+}
+
+extern "C" size_t sifar_chain_ring_stride(int dtype, size_t n)
+{
+    if (dtype != SIFAR_BF16 && dtype != SIFAR_F32) return 0;
+    return (n * elem_size(dtype) + 255) / 256 * 256;
+}
+
+template <int DT>
+static cudaError_t launch_produce_dt(int mode, int grid, cudaStream_t s, const ProduceArgs &a)
+{
+    switch (mode) {
+    case SIFAR_BARRIER_ONESHOT: k_produce<DT, SIFAR_BARRIER_ONESHOT><<<grid, kProdThreads, 0, s>>>(a); break;
+    case SIFAR_DUALBUF:         k_produce<DT, SIFAR_DUALBUF><<<grid, kProdThreads, 0, s>>>(a); break;
+    case SIFAR_SPECULATIVE:     k_produce<DT, SIFAR_SPECULATIVE><<<grid, kProdThreads, 0, s>>>(a); break;
+    default:                    k_produce<DT, kModeNoAllreduce><<<grid, kProdThreads, 0, s>>>(a); break;
+    }
+    return cudaGetLastError();
+}
+
+static const void *chain_rank_buffer(const sifar_ctx *c, int mode, uint32_t e, int r)
+{
+    if (mode == SIFAR_BARRIER_ONESHOT) return c->plain_buf(0, r);
+    if (mode == SIFAR_SPECULATIVE) return c->slot_buf((int)(e & 1u), r);
+    return c->plain_buf((int)(e & 1u), r);          /* DUALBUF and the no-all-reduce floor */
+}
+
+/* Enqueue one run (steps steps starting at step first_t) as P producer streams + one reducer stream forked from `origin`. */
+static int enqueue_run(sifar_chain *ch, cudaStream_t origin, uint32_t first_t)
+{
+    sifar_ctx *c = ch->ctx;
+    const int P = c->P;
+    const bool no_ar = (ch->mode == kModeNoAllreduce);
+    SIFAR_CUDA(cudaEventRecord(ch->ev_fork, origin));
+    for (int r = 0; r < P; ++r) SIFAR_CUDA(cudaStreamWaitEvent(ch->prod[r], ch->ev_fork, 0));
+    if (!no_ar) SIFAR_CUDA(cudaStreamWaitEvent(ch->red, ch->ev_fork, 0));
+
+    const size_t units = (ch->mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, ch->n)
+                                                         : (ch->n * elem_size(c->dtype) + 15) / 16;
+    size_t pgrid = (units + kProdThreads - 1) / kProdThreads;
+    const size_t cap = (size_t)c->sm_count * 2;
+    if (pgrid > cap) pgrid = cap;
+
+    for (int s = 0; s < ch->steps; ++s) {
+        const uint32_t t = first_t + (uint32_t)s;
+        const uint32_t e = ch->base_epoch + t;
+        for (int r = 0; r < P; ++r) {
+            if (s > 0 && !no_ar) SIFAR_CUDA(cudaStreamWaitEvent(ch->prod[r], ch->ev_step[s - 1], 0));
+            ProduceArgs a;
+            memset(&a, 0, sizeof a);
+            a.st = c->d_state; a.host_status = c->d_status_alias; a.timeout_ns = c->timeout_ns;
+            a.w = ch->w; a.rank = (uint32_t)r; a.n = ch->n;
+            a.dst = const_cast<void *>(chain_rank_buffer(c, ch->mode, e, r));
+            a.prev = no_ar ? chain_rank_buffer(c, ch->mode, e - 1u, r)
+                           : ch->ring + (size_t)((t + ch->ring_len - 2u) % ch->ring_len) * ch->ring_stride;
+            a.base_epoch = ch->base_epoch; a.parity = e & 1u;
+            a.t_fixed = no_ar ? t : 0u;
+            cudaError_t err = (c->dtype == SIFAR_BF16)
+                ? launch_produce_dt<SIFAR_BF16>(ch->mode, (int)pgrid, ch->prod[r], a)
+                : launch_produce_dt<SIFAR_F32>(ch->mode, (int)pgrid, ch->prod[r], a);
+            SIFAR_CUDA(err);
+        }
+        if (!no_ar) {
+            ReduceLaunch rl;
+            memset(&rl, 0, sizeof rl);
+            for (int r = 0; r < P; ++r) rl.src[r] = chain_rank_buffer(c, ch->mode, e, r);
+            rl.out = ch->ring + (size_t)((t - 1u) % ch->ring_len) * ch->ring_stride;
+            rl.n = ch->n; rl.mode = ch->mode; rl.parity = e & 1u;
+            int rc = launch_reduce(c, rl, ch->red);
+            if (rc) return rc;
+            SIFAR_CUDA(cudaEventRecord(ch->ev_step[s], ch->red));
+        }
+    }
+    for (int r = 0; r < P; ++r) {
+        SIFAR_CUDA(cudaEventRecord(ch->ev_join[r], ch->prod[r]));
+        SIFAR_CUDA(cudaStreamWaitEvent(origin, ch->ev_join[r], 0));
+    }
+    if (!no_ar) {
+        SIFAR_CUDA(cudaEventRecord(ch->ev_join[P], ch->red));
+        SIFAR_CUDA(cudaStreamWaitEvent(origin, ch->ev_join[P], 0));
+    }
+    return SIFAR_OK;
+}
+
+template <int DT, int P>
+static const void *chain_kernel_p(int mode)
+{
+    switch (mode) {
+    case SIFAR_BARRIER_ONESHOT: return (const void *)k_chain<DT, P, SIFAR_BARRIER_ONESHOT>;
+    case SIFAR_DUALBUF:         return (const void *)k_chain<DT, P, SIFAR_DUALBUF>;
+    case SIFAR_SPECULATIVE:     return (const void *)k_chain<DT, P, SIFAR_SPECULATIVE>;
+    default:                    return (const void *)k_chain<DT, P, kModeNoAllreduce>;
+    }
+}
+
+template <int DT>
+static const void *chain_kernel_dt(int P, int mode)
+{
+    switch (P) {
+    case 1: return chain_kernel_p<DT, 1>(mode);
+    case 2: return chain_kernel_p<DT, 2>(mode);
+    case 3: return chain_kernel_p<DT, 3>(mode);
+    case 4: return chain_kernel_p<DT, 4>(mode);
+    case 5: return chain_kernel_p<DT, 5>(mode);
+    case 6: return chain_kernel_p<DT, 6>(mode);
+    case 7: return chain_kernel_p<DT, 7>(mode);
+    default: return chain_kernel_p<DT, 8>(mode);
+    }
+}
+
+static const void *chain_kernel(const sifar_chain *ch)
+{
+    return ch->ctx->dtype == SIFAR_BF16 ? chain_kernel_dt<SIFAR_BF16>(ch->ctx->P, ch->mode)
+                                        : chain_kernel_dt<SIFAR_F32>(ch->ctx->P, ch->mode);
+}
+
+static void chain_free(sifar_chain *ch)
+{
+    if (!ch) return;
+    for (int r = 0; r < kMaxRanks; ++r) if (ch->prod[r]) cudaStreamDestroy(ch->prod[r]);
+    if (ch->red) cudaStreamDestroy(ch->red);
+    if (ch->ev_fork) cudaEventDestroy(ch->ev_fork);
+    for (int r = 0; r <= kMaxRanks; ++r) if (ch->ev_join[r]) cudaEventDestroy(ch->ev_join[r]);
+    for (cudaEvent_t e : ch->ev_step) if (e) cudaEventDestroy(e);
+    if (ch->exec) cudaGraphExecDestroy(ch->exec);
+    if (ch->graph) cudaGraphDestroy(ch->graph);
+    if (ch->d_cs) cudaFree(ch->d_cs);
+    if (ch->d_chunks) cudaFree(ch->d_chunks);
+    if (ch->d_stamps) cudaFree(ch->d_stamps);
+    if (ch->d_retry_steps) cudaFree(ch->d_retry_steps);
+    delete ch;
+}
+
+static int chain_setup_persistent(sifar_chain *ch)
+{
+    sifar_ctx *c = ch->ctx;
+    const int roles = (ch->mode == kModeNoAllreduce) ? c->P : c->P + 1;
+    const size_t units = (ch->mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, ch->n)
+                                                         : (ch->n * elem_size(c->dtype) + 15) / 16;
+    int per_sm = 0;
+    SIFAR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, chain_kernel(ch), kChainThreads, 0));
+    const size_t resident = (size_t)per_sm * c->sm_count;
+    /* leave half of the machine free: the chain stands for a few operators of a forward pass, not all of it */
+    const size_t budget = resident / 2 > (size_t)roles ? resident / 2 : (size_t)roles;
+    uint32_t K = 1;
+    size_t C = (units + kChainThreads - 1) / kChainThreads;
+    while (C * roles > budget) {
+        ++K;
+        C = (units + (size_t)kChainThreads * K - 1) / ((size_t)kChainThreads * K);
+    }
+    ch->K = K; ch->C = (uint32_t)C; ch->grid = (int)(C * roles);
+    SIFAR_CUDA(cudaMalloc(&ch->d_cs, sizeof(ChainDev)));
+    SIFAR_CUDA(cudaMalloc(&ch->d_chunks, sizeof(ChunkFlags) * C));
+    SIFAR_CUDA(cudaMalloc(&ch->d_stamps, sizeof(unsigned long long) * (ch->steps + 1)));
+    SIFAR_CUDA(cudaMalloc(&ch->d_retry_steps, sizeof(uint32_t) * ch->steps));
+    SIFAR_CUDA(cudaMemset(ch->d_cs, 0, sizeof(ChainDev)));
+    SIFAR_CUDA(cudaMemset(ch->d_chunks, 0, sizeof(ChunkFlags) * C));
+    SIFAR_CUDA(cudaMemset(ch->d_stamps, 0, sizeof(unsigned long long) * (ch->steps + 1)));
+    SIFAR_CUDA(cudaMemset(ch->d_retry_steps, 0, sizeof(uint32_t) * ch->steps));
+    return SIFAR_OK;
+}
+
+extern "C" sifar_chain *sifar_chain_create(sifar_ctx *c, const sifar_workload *w, size_t n, int mode, int impl,
+                                           void *out_ring, int ring_len, int steps_per_run)
+{
+    if (!c || !valid_workload(w) || n == 0 || n > c->max_elems || mode < 0 || mode > kModeNoAllreduce ||
+        impl < 0 || impl > SIFAR_CHAIN_PERSISTENT || !out_ring || ((uintptr_t)out_ring & 15u) || ring_len < 2 ||
+        steps_per_run < 2 || (steps_per_run & 1) || steps_per_run % ring_len != 0) {
+        set_error("sifar_chain_create: bad argument (need 1 <= n <= max_elems, ring_len >= 2 dividing an even "
+                  "steps_per_run, delay_max_ns <= %u)", kMaxDelayNs);
+        return nullptr;
+    }
+    if (*c->h_status != 0) { set_error("sifar_chain_create: context carries a device error"); return nullptr; }
+    if ((uint64_t)c->h_epoch + (uint64_t)steps_per_run >= kEpochLimit) {
+        set_error("sifar_chain_create: call numbers exhausted");
+        return nullptr;
+    }
+    sifar_chain *ch = new (std::nothrow) sifar_chain();
+    if (!ch) { set_error("sifar_chain_create: out of host memory"); return nullptr; }
+    ch->ctx = c; ch->w = *w; ch->n = n; ch->mode = mode; ch->impl = impl;
+    ch->ring = (char *)out_ring; ch->ring_len = ring_len;
+    ch->ring_stride = sifar_chain_ring_stride(c->dtype, n);
+    ch->steps = steps_per_run; ch->base_epoch = c->h_epoch; ch->runs = 0;
+    cudaSetDevice(c->device);
+    int rc = SIFAR_OK;
+    auto setup = [&]() -> int {
+        if (impl == SIFAR_CHAIN_PERSISTENT) {
+            int coop = 0;
+            SIFAR_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
+            if (!coop) { set_error("sifar_chain_create: device lacks cooperative launch"); return SIFAR_ERR_CUDA; }
+            ch->launches_per_run = 1;
+            return chain_setup_persistent(ch);
+        }
+        for (int r = 0; r < c->P; ++r) SIFAR_CUDA(cudaStreamCreateWithFlags(&ch->prod[r], cudaStreamNonBlocking));
+        SIFAR_CUDA(cudaStreamCreateWithFlags(&ch->red, cudaStreamNonBlocking));
+        SIFAR_CUDA(cudaEventCreateWithFlags(&ch->ev_fork, cudaEventDisableTiming));
+        for (int r = 0; r <= c->P; ++r) SIFAR_CUDA(cudaEventCreateWithFlags(&ch->ev_join[r], cudaEventDisableTiming));
+        ch->ev_step.assign((size_t)ch->steps, nullptr);
+        for (int s = 0; s < ch->steps; ++s) SIFAR_CUDA(cudaEventCreateWithFlags(&ch->ev_step[s], cudaEventDisableTiming));
+        ch->launches_per_run = ch->steps * (c->P + (mode == kModeNoAllreduce ? 0 : 1));
+        if (impl == SIFAR_CHAIN_GRAPH) {
+            /* capture one run; every later replay finds the same parities because steps_per_run is even */
+            cudaStream_t cap;
+            SIFAR_CUDA(cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking));
+            cudaError_t err = cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal);
+            int erc = SIFAR_OK;
+            if (err == cudaSuccess) {
+                erc = enqueue_run(ch, cap, 1u);
+                err = cudaStreamEndCapture(cap, &ch->graph);
+            }
+            cudaStreamDestroy(cap);
+            if (erc) return erc;
+            SIFAR_CUDA(err);
+            SIFAR_CUDA(cudaGraphInstantiate(&ch->exec, ch->graph, 0));
+        }
+        return SIFAR_OK;
+    };
+    rc = setup();
+    if (rc) { cudaGetLastError(); chain_free(ch); return nullptr; }
+    return ch;
+}
+
+extern "C" int sifar_chain_run(sifar_chain *ch, void *stream)
+{
+    if (!ch) { set_error("sifar_chain_run: NULL chain"); return SIFAR_ERR_INVALID; }
+    sifar_ctx *c = ch->ctx;
+    const int s0 = *c->h_status;
+    if (s0) { set_error("sifar_chain_run: context carries device status %d", s0); return s0; }
+    const bool no_ar = (ch->mode == kModeNoAllreduce);
+    const uint32_t expect = ch->base_epoch + (no_ar ? 0u : ch->runs * (uint32_t)ch->steps);
+    if (c->h_epoch != expect) {
+        set_error("sifar_chain_run: the context was used outside the chain (call number %u, expected %u)",
+                  c->h_epoch, expect);
+        return SIFAR_ERR_EPOCH;
+    }
+    if ((uint64_t)c->h_epoch + (uint64_t)ch->steps >= kEpochLimit) {
+        set_error("sifar_chain_run: call numbers exhausted");
+        return SIFAR_ERR_EPOCH;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    const uint32_t first_t = ch->runs * (uint32_t)ch->steps + 1u;
+    if (ch->impl == SIFAR_CHAIN_STREAMS) {
+        int rc = enqueue_run(ch, s, first_t);
+        if (rc) return rc;
+    } else if (ch->impl == SIFAR_CHAIN_GRAPH) {
+        SIFAR_CUDA(cudaGraphLaunch(ch->exec, s));
+    } else {
+        PersistArgs a;
+        memset(&a, 0, sizeof a);
+        a.st = c->d_state; a.host_status = c->d_status_alias; a.timeout_ns = c->timeout_ns;
+        a.w = ch->w; a.n = ch->n;
+        a.plain = c->d_plain; a.plain_stride = c->plain_stride;
+        a.slots = c->d_slots; a.slot_stride = c->slot_stride;
+        a.ring = ch->ring; a.ring_stride = ch->ring_stride; a.ring_len = (uint32_t)ch->ring_len;
+        a.e0 = no_ar ? ch->base_epoch + ch->runs * (uint32_t)ch->steps : c->h_epoch;
+        a.base_epoch = ch->base_epoch; a.steps = (uint32_t)ch->steps;
+        a.C = ch->C; a.K = ch->K;
+        a.bottom_base = ch->runs * (uint32_t)ch->steps * ch->C;
+        a.exit_base = ch->runs * (uint32_t)ch->grid;
+        a.cs = ch->d_cs; a.chunks = ch->d_chunks; a.stamps = ch->d_stamps; a.retry_steps = ch->d_retry_steps;
+        void *params[] = {&a};
+        SIFAR_CUDA(cudaLaunchCooperativeKernel(chain_kernel(ch), dim3((unsigned)ch->grid), dim3(kChainThreads),
+                                               params, 0, s));
+    }
+    ch->runs += 1;
+    if (!no_ar) c->h_epoch += (uint32_t)ch->steps;
+    if (ch->mode == SIFAR_BARRIER_ONESHOT) c->last_mode0_epoch = c->h_epoch;
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_chain_stamps(sifar_chain *ch, unsigned long long *stamps)
+{
+    if (!ch || !stamps || ch->impl != SIFAR_CHAIN_PERSISTENT) {
+        set_error("sifar_chain_stamps: needs a persistent chain and a destination");
+        return SIFAR_ERR_INVALID;
+    }
+    SIFAR_CUDA(cudaDeviceSynchronize());
+    SIFAR_CUDA(cudaMemcpy(stamps, ch->d_stamps, sizeof(unsigned long long) * (ch->steps + 1), cudaMemcpyDeviceToHost));
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_chain_launches_per_run(sifar_chain *ch)
+{
+    return ch ? ch->launches_per_run : 0;
+}
+
+extern "C" int sifar_chain_destroy(sifar_chain *ch)
+{
+    if (!ch) return SIFAR_OK;
+    cudaSetDevice(ch->ctx->device);
+    cudaError_t e = cudaDeviceSynchronize();
+    chain_free(ch);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+    return SIFAR_OK;
+}
+
+static int probe_launch(const sifar_workload *w, int rank, unsigned t, int dtype, const void *prev, void *dst,
+                        size_t n, void *stream)
+{
+    if (!valid_workload(w) || rank < 0 || (dtype != SIFAR_BF16 && dtype != SIFAR_F32) || !dst ||
+        ((uintptr_t)dst & 15u) || (t > 1 && (!prev || ((uintptr_t)prev & 15u))) || t == 0) {
+        set_error("sifar_workload probe: bad argument");
+        return SIFAR_ERR_INVALID;
+    }
+    if (n == 0) return SIFAR_OK;
+    size_t grid = (n / 8 + 255) / 256;
+    if (grid < 1) grid = 1;
+    if (grid > 1184) grid = 1184;
+    if (dtype == SIFAR_BF16)
+        k_probe<SIFAR_BF16><<<(int)grid, 256, 0, (cudaStream_t)stream>>>(*w, (uint32_t)rank, t, prev, dst, n);
+    else
+        k_probe<SIFAR_F32><<<(int)grid, 256, 0, (cudaStream_t)stream>>>(*w, (uint32_t)rank, t, prev, dst, n);
+    SIFAR_CUDA(cudaGetLastError());
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_workload_first(const sifar_workload *w, int rank, int dtype, void *dst, size_t n, void *stream)
+{
+    return probe_launch(w, rank, 1u, dtype, nullptr, dst, n, stream);
+}
+
+extern "C" int sifar_workload_next(const sifar_workload *w, int rank, unsigned t, int dtype, const void *prev_out,
+                                   void *dst, size_t n, void *stream)
+{
+    if (t < 2) { set_error("sifar_workload_next: t must be >= 2"); return SIFAR_ERR_INVALID; }
+    return probe_launch(w, rank, t, dtype, prev_out, dst, n, stream);
+}
+
+extern "C" int sifar_workload_delays(const sifar_workload *w, int P, unsigned t, unsigned *host_out)
+{
+    if (!w || P < 1 || P > 32 || !host_out) { set_error("sifar_workload_delays: bad argument"); return SIFAR_ERR_INVALID; }
+    unsigned *d = nullptr;
+    SIFAR_CUDA(cudaMalloc(&d, sizeof(unsigned) * 32));
+    k_delays<<<1, 32>>>(*w, P, t, d);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaMemcpy(host_out, d, sizeof(unsigned) * P, cudaMemcpyDeviceToHost);
+    cudaFree(d);
+    SIFAR_CUDA(e);
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_spin(unsigned ns, void *stream)
+{
+    if (ns > 50000000u) { set_error("sifar_spin: at most 50 ms"); return SIFAR_ERR_INVALID; }
+    k_spin<<<1, 1, 0, (cudaStream_t)stream>>>(ns);
+    SIFAR_CUDA(cudaGetLastError());
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_tear_check(unsigned nslots, unsigned rounds, unsigned long long *host_torn,
+                                unsigned long long *host_reads)
+{
+    if (nslots == 0 || rounds == 0 || rounds > 100000 || !host_torn || !host_reads) {
+        set_error("sifar_tear_check: bad argument");
+        return SIFAR_ERR_INVALID;
+    }
+    int dev = 0, sms = 0;
+    SIFAR_CUDA(cudaGetDevice(&dev));
+    SIFAR_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    uint4 *slots = nullptr;
+    unsigned long long *counters = nullptr;
+    SIFAR_CUDA(cudaMalloc(&slots, (size_t)nslots * 16));
+    cudaError_t e = cudaMalloc(&counters, 16);
+    if (e == cudaSuccess) e = cudaMemset(slots, 0, (size_t)nslots * 16);
+    if (e == cudaSuccess) e = cudaMemset(counters, 0, 16);
+    if (e == cudaSuccess) {
+        /* writers and readers must overlap in time: launch them as one cooperative grid, one CTA per SM */
+        unsigned writers = (unsigned)sms / 2;
+        unsigned long long *torn = counters, *reads = counters + 1;
+        void *params[] = {&slots, &nslots, &rounds, &writers, &torn, &reads};
+        e = cudaLaunchCooperativeKernel((const void *)k_tear, dim3((unsigned)sms), dim3(256), params, 0, 0);
+    }
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    unsigned long long h[2] = {0, 0};
+    if (e == cudaSuccess) e = cudaMemcpy(h, counters, 16, cudaMemcpyDeviceToHost);
+    cudaFree(slots);
+    if (counters) cudaFree(counters);
+    SIFAR_CUDA(e);
+    *host_torn = h[0];
+    *host_reads = h[1];
+    return SIFAR_OK;
+}
