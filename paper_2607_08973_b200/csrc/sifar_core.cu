@@ -24,6 +24,7 @@
  */
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -63,6 +64,7 @@ struct ReduceArgs {
     unsigned long long timeout_ns;
     uint32_t parity;
     uint32_t check_parity;
+    uint32_t poll_wide;      /* speculative: re-load all stale ranks per round (else one at a time) */
 };
 
 struct PackArgs {
@@ -225,7 +227,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
         for (int u = 0; u < U; ++u) {
             const size_t s = base + (size_t)u * kThreads;
             if (s >= nslots) continue;
-            if (!validate_slot<P>(x[u], a.src, s, e, a.timeout_ns, reloads)) {
+            if (!validate_slot<P>(x[u], a.src, s, e, a.timeout_ns, a.poll_wide != 0u, reloads)) {
                 fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
                 alive = false;
                 break;
@@ -392,6 +394,16 @@ static cudaError_t launch_reduce_dt(int P, int mode, int grid, cudaStream_t s, c
     }
 }
 
+}  /* namespace sifar */
+
+/* Wide polling while the whole grid's polling volume per round stays small (see validate_slot). */
+uint32_t sifar::poll_wide_for(const sifar_ctx *ctx, size_t n)
+{
+    return slots_for(ctx->dtype, n) * (size_t)ctx->P <= ctx->poll_wide_max ? 1u : 0u;
+}
+
+namespace sifar {
+
 static int unroll_for(int P) { return P <= 2 ? 4 : P <= 4 ? 2 : 1; }
 
 int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
@@ -411,6 +423,7 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
     a.timeout_ns = ctx->timeout_ns;
     a.parity = rl.parity;
     a.check_parity = (rl.mode != SIFAR_BARRIER_ONESHOT);
+    a.poll_wide = poll_wide_for(ctx, rl.n);
     size_t units = (rl.mode == SIFAR_SPECULATIVE) ? slots_for(ctx->dtype, rl.n)
                                                   : (rl.n * elem_size(ctx->dtype) + 15) / 16;
     const int grid = reduce_grid(ctx, units, unroll_for(ctx->P));
@@ -477,6 +490,8 @@ extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
     memset(c, 0, sizeof *c);
     c->P = P; c->dtype = dtype; c->max_elems = max_elems;
     c->timeout_ns = 200000ull * 1000ull;
+    c->poll_wide_max = 16384;
+    if (const char *env = getenv("SIFAR_POLL_WIDE_MAX")) c->poll_wide_max = (size_t)strtoull(env, nullptr, 10);
     cudaError_t e = cudaGetDevice(&c->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
     c->plain_stride = round_up(max_elems * elem_size(dtype), 256);

@@ -81,6 +81,7 @@ struct sifar_ctx {
     uint32_t h_epoch;                /* calls enqueued so far                            */
     uint32_t last_mode0_epoch;       /* last BARRIER_ONESHOT call (0: none): whose done flags a producer waits for */
     unsigned long long timeout_ns;
+    size_t poll_wide_max;            /* speculative: wide polling up to this many (slot, rank) pairs per call */
     /* staging for sifar_allreduce_host, allocated on first use */
     char *d_stage_in;
     char *d_stage_out;
@@ -113,6 +114,7 @@ struct ReduceLaunch {
 };
 
 int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream);
+uint32_t poll_wide_for(const sifar_ctx *ctx, size_t n);
 
 }  /* namespace sifar */
 #endif

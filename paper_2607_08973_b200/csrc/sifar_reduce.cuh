@@ -14,32 +14,42 @@ namespace sifar {
 /* bounded waits                                                             */
 /* ------------------------------------------------------------------------ */
 
+/*
+ * Reading %globaltimer is slow next to an L2 round trip, so the time limit is
+ * only looked at every kPollsPerClockCheck failed polls; a poll costs at least
+ * one trip to the L2, which keeps the overshoot to a few tens of microseconds.
+ */
+constexpr unsigned kPollsPerClockCheck = 64;
+
+struct Deadline {
+    unsigned long long t0 = 0;
+    unsigned polls = 0;
+    /* Call after a failed poll; true once the limit has passed. */
+    __device__ __forceinline__ bool expired(unsigned long long timeout_ns)
+    {
+        if ((++polls % kPollsPerClockCheck) != 0u) return false;
+        const unsigned long long now = globaltimer_ns();
+        if (t0 == 0) { t0 = now; return false; }
+        return now - t0 > timeout_ns;
+    }
+};
+
 /* Bounded poll of a flag until it equals `want` (acquire).  Returns the number of failed polls, or -1 on time-out. */
 __device__ __forceinline__ int wait_flag_eq(const uint32_t *flag, uint32_t want, unsigned long long timeout_ns)
 {
-    int polls = 0;
-    unsigned long long t0 = 0;
-    while (ld_acquire_u32(flag) != want) {
-        ++polls;
-        unsigned long long now = globaltimer_ns();
-        if (t0 == 0) t0 = now;
-        else if (now - t0 > timeout_ns) return -1;
-    }
-    return polls;
+    Deadline d;
+    while (ld_acquire_u32(flag) != want)
+        if (d.expired(timeout_ns)) return -1;
+    return (int)d.polls;
 }
 
-/* Same for "flag - base is in [0, 2^31)", i.e. flag has reached `base` (call numbers never wrap inside a context's life). */
+/* Same until the flag has reached `base` (call numbers never wrap inside a context's life). */
 __device__ __forceinline__ int wait_flag_ge(const uint32_t *flag, uint32_t base, unsigned long long timeout_ns)
 {
-    int polls = 0;
-    unsigned long long t0 = 0;
-    while (ld_acquire_u32(flag) < base) {
-        ++polls;
-        unsigned long long now = globaltimer_ns();
-        if (t0 == 0) t0 = now;
-        else if (now - t0 > timeout_ns) return -1;
-    }
-    return polls;
+    Deadline d;
+    while (ld_acquire_u32(flag) < base)
+        if (d.expired(timeout_ns)) return -1;
+    return (int)d.polls;
 }
 
 /* ------------------------------------------------------------------------ */
@@ -87,33 +97,40 @@ template <int P> struct Unroll { static constexpr int value = (P <= 2) ? 4 : (P 
 /*
  * x[r] holds rank r's slot `s` as first loaded.  A slot counts iff its tag equals
  * the call number e (Section 4.2: validation after the speculative read).  On
- * mis-speculation only the stale ranks of this slot are loaded again, with a
- * short back-off, until every tag matches or the time limit passes.  Returns
- * false on time-out.  `reloads` counts the extra loads.
+ * mis-speculation only the stale ranks of this slot are loaded again until
+ * every tag matches or the time limit passes.  Returns false on time-out.
+ * `reloads` counts the extra loads.
+ *
+ * Two polling shapes.  wide: every stale rank is re-loaded each round; the last
+ * arrival is seen one L2 round trip later, at P loads per waiting thread and
+ * round.  narrow: only the lowest stale rank is polled; when it turns valid one
+ * wide round follows.  Narrow costs one more round trip after the last arrival
+ * but keeps the polling traffic of a large waiting grid from starving the
+ * producers' stores of L2 bandwidth.
  */
 template <int P>
 __device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const *src, size_t s, uint32_t e,
-                                              unsigned long long timeout_ns, unsigned &reloads)
+                                              unsigned long long timeout_ns, bool wide, unsigned &reloads)
 {
     uint32_t stale = 0;
 #pragma unroll
     for (int r = 0; r < P; ++r) stale |= (uint32_t)(x[r].w != e) << r;
     if (stale == 0u) return true;
-    const unsigned long long t0 = globaltimer_ns();
-    unsigned spins = 0;
+    Deadline d;
+    bool burst = wide;
     do {
+        /* issue every pending load before looking at any result, so that the re-loads overlap */
+        const uint32_t pending = burst ? stale : (stale & (0u - stale));
 #pragma unroll
-        for (int r = 0; r < P; ++r) {
-            if (stale & (1u << r)) {
-                x[r] = ld_slot(src[r] + s);
-                ++reloads;
-                if (x[r].w == e) stale &= ~(1u << r);
-            }
-        }
-        if (stale) {
-            if (globaltimer_ns() - t0 > timeout_ns) return false;
-            if (++spins > 8) __nanosleep(spins > 64 ? 200 : 40);
-        }
+        for (int r = 0; r < P; ++r)
+            if (pending & (1u << r)) x[r] = ld_slot(src[r] + s);
+        const uint32_t before = stale;
+#pragma unroll
+        for (int r = 0; r < P; ++r)
+            if ((pending & (1u << r)) && x[r].w == e) stale &= ~(1u << r);
+        reloads += __popc(pending);
+        burst = wide || (!burst && stale != before);     /* narrow: the polled rank arrived, look at all others once */
+        if (stale && d.expired(timeout_ns)) return false;
     } while (stale);
     return true;
 }

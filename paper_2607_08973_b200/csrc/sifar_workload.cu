@@ -120,14 +120,47 @@ __device__ __forceinline__ float next_value(const Gen &g, uint32_t i, float prev
 }
 
 /*
- * One unit of a rank's partial: NW 32-bit words starting at element i0 (bf16: two
- * elements per word), elements at or past n are zero.  `prev` is out^{t-1}
- * (ignored when `first`); it is read with strong loads because inside the
- * persistent kernel it was written by another CTA of the same launch.
+ * A unit of a rank's partial is NW 32-bit words starting at element i0 (bf16: two
+ * elements per word); elements at or past n are zero.  It is computed in two
+ * halves so that the half that does not depend on the previous result can run
+ * while that result is still being reduced:
+ *   unit_noise()   the seeded part: the whole first partial, or sigma * z
+ *                  (kinds 0, 2), or the integer k (kind 1);
+ *   unit_combine() loads out^{t-1} and applies the update rule.
+ * out^{t-1} is read with strong loads: inside the persistent kernel it was
+ * written by another CTA of the same launch.
  */
 template <int DT, int NW>
-__device__ __forceinline__ void produce_words(const Gen &g, bool first, const void *prev, size_t i0, size_t n,
-                                              uint32_t (&w)[NW])
+__device__ __forceinline__ void unit_noise(const Gen &g, bool first, size_t i0, size_t n,
+                                           float (&z)[NW * ((DT == SIFAR_BF16) ? 2 : 1)])
+{
+    constexpr int NE = NW * ((DT == SIFAR_BF16) ? 2 : 1);
+#pragma unroll
+    for (int k = 0; k < NE; ++k) {
+        const size_t i = i0 + k;
+        z[k] = 0.0f;
+        if (i < n) {
+            if (first) z[k] = first_value(g, (uint32_t)i);
+            else if (g.kind == 1) z[k] = (float)gen_int129(g, (uint32_t)i);
+            else z[k] = __fmul_rn((g.kind == 2) ? gen_uniform(g, (uint32_t)i) : gen_gauss(g, (uint32_t)i), g.sigma);
+        }
+    }
+}
+
+__device__ __forceinline__ float apply_update(const Gen &g, bool first, float prev, float z)
+{
+    if (first) return z;
+    if (g.kind == 1) {
+        int32_t v = ((int32_t)prev + (int32_t)z) % 129;
+        if (v < 0) v += 129;
+        return (float)(v - 64);
+    }
+    return __fadd_rn(__fmul_rn(prev, g.scale), z);
+}
+
+template <int DT, int NW>
+__device__ __forceinline__ void unit_combine(const Gen &g, bool first, const void *prev, size_t i0, size_t n,
+                                             const float (&z)[NW * ((DT == SIFAR_BF16) ? 2 : 1)], uint32_t (&w)[NW])
 {
     constexpr int EPW = (DT == SIFAR_BF16) ? 2 : 1;
     uint32_t pw[NW];
@@ -157,20 +190,25 @@ __device__ __forceinline__ void produce_words(const Gen &g, bool first, const vo
     for (int j = 0; j < NW; ++j) {
         if (DT == SIFAR_BF16) {
             const size_t ia = i0 + 2 * j, ib = ia + 1;
-            float a = 0.0f, b = 0.0f;
-            if (ia < n) a = first ? first_value(g, (uint32_t)ia) : next_value(g, (uint32_t)ia, bf16lo_to_f32(pw[j]));
-            if (ib < n) b = first ? first_value(g, (uint32_t)ib) : next_value(g, (uint32_t)ib, bf16hi_to_f32(pw[j]));
+            const float a = (ia < n) ? apply_update(g, first, bf16lo_to_f32(pw[j]), z[2 * j]) : 0.0f;
+            const float b = (ib < n) ? apply_update(g, first, bf16hi_to_f32(pw[j]), z[2 * j + 1]) : 0.0f;
             w[j] = f32x2_to_bf16x2(a, b);
             if (ia >= n) w[j] = 0u;
             else if (ib >= n) w[j] &= 0xFFFFu;
         } else {
             const size_t ia = i0 + j;
-            w[j] = 0u;
-            if (ia < n)
-                w[j] = __float_as_uint(first ? first_value(g, (uint32_t)ia)
-                                             : next_value(g, (uint32_t)ia, __uint_as_float(pw[j])));
+            w[j] = (ia < n) ? __float_as_uint(apply_update(g, first, __uint_as_float(pw[j]), z[j])) : 0u;
         }
     }
+}
+
+template <int DT, int NW>
+__device__ __forceinline__ void produce_words(const Gen &g, bool first, const void *prev, size_t i0, size_t n,
+                                              uint32_t (&w)[NW])
+{
+    float z[NW * ((DT == SIFAR_BF16) ? 2 : 1)];
+    unit_noise<DT, NW>(g, first, i0, n, z);
+    unit_combine<DT, NW>(g, first, prev, i0, n, z, w);
 }
 
 /* Busy-wait `ns` nanoseconds on the global timer (ns is small and bounded by the caller). */
@@ -318,6 +356,7 @@ struct PersistArgs {
     uint32_t C;                     /* chunks = reducer CTAs               */
     uint32_t K;                     /* units per thread and step           */
     uint32_t bottom_base, exit_base;
+    uint32_t poll_wide;
     ChainDev *cs;
     ChunkFlags *chunks;
     unsigned long long *stamps;     /* steps + 1                           */
@@ -331,15 +370,12 @@ template <bool GE>
 __device__ __forceinline__ bool chain_wait(const uint32_t *flag, uint32_t want, DevState *st, int *host_status,
                                            unsigned long long timeout_ns)
 {
-    unsigned long long t0 = 0;
-    unsigned polls = 0;
+    Deadline d;
     for (;;) {
         const uint32_t v = ld_acquire_u32(flag);
         if (GE ? (v >= want) : (v == want)) return true;
-        const unsigned long long now = globaltimer_ns();
-        if (t0 == 0) t0 = now;
-        else if (now - t0 > timeout_ns) { fail(st, host_status, SIFAR_ERR_TIMEOUT); return false; }
-        if ((++polls & 63u) == 0u && ld_relaxed_u32(&st->status) != 0u) return false;
+        if (d.expired(timeout_ns)) { fail(st, host_status, SIFAR_ERR_TIMEOUT); return false; }
+        if ((d.polls % kPollsPerClockCheck) == 0u && ld_relaxed_u32(&st->status) != 0u) return false;
     }
 }
 
@@ -359,6 +395,9 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
     const size_t nunits = (n + EPU - 1) / EPU;
     const size_t unit0 = (size_t)chunk * kChainThreads * a.K + threadIdx.x;
     __shared__ int s_ok;
+    __shared__ int s_retried[2];
+    if (threadIdx.x < 2) s_retried[threadIdx.x] = 0;
+    __syncthreads();
     unsigned reloads = 0;
     bool alive = true;
     const bool stamper = (blockIdx.x == 0);     /* reducer of chunk 0 (or rank 0's producer of chunk 0 without all-reduce) */
@@ -402,7 +441,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                 for (int r = 0; r < P; ++r) x[r] = ld_slot(src[r] + u);
                 if (MODE == SIFAR_SPECULATIVE) {
                     const unsigned before = reloads;
-                    if (!validate_slot<P>(x, src, u, e, a.timeout_ns, reloads)) {
+                    if (!validate_slot<P>(x, src, u, e, a.timeout_ns, a.poll_wide != 0u, reloads)) {
                         fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
                         alive = false;
                         break;
@@ -413,10 +452,16 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                     store_vec_result<DT>(ring_row, u, n, sum_vec<DT, P>(x, true));
                 }
             }
-            if (MODE == SIFAR_SPECULATIVE && retried) st_relaxed_u32(&a.retry_steps[s], 1u);
+            /* "somebody in this CTA re-loaded a slot": two alternating words, so that clearing one after the
+               barrier of step s cannot race with the marks of step s + 1 */
+            if (MODE == SIFAR_SPECULATIVE && retried) s_retried[s & 1u] = 1;
             if (!__syncthreads_and(alive)) { alive = false; break; }
             if (threadIdx.x == 0) {
                 st_release_u32(&cf->ready, e);                 /* result chunk published */
+                if (MODE == SIFAR_SPECULATIVE && s_retried[s & 1u]) {
+                    s_retried[s & 1u] = 0;
+                    st_relaxed_u32(&a.retry_steps[s], 1u);
+                }
                 if (stamper) a.stamps[s + 1u] = globaltimer_ns();
                 if (MODE == SIFAR_BARRIER_ONESHOT) {
                     /* bottom barrier, reducer side: last CTA to finish reading releases the done flags */
@@ -427,6 +472,19 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
             }
         } else {
             /* ---------------- rank `rank`, chunk `chunk` of the next operation ---------------- */
+            constexpr int NW = (MODE == SIFAR_SPECULATIVE) ? 3 : 4;
+            constexpr int NE = NW * ((DT == SIFAR_BF16) ? 2 : 1);
+            const Gen g = make_gen(a.w, rank, t);
+            const bool first = (t == 1u);
+            /* the seeded half of the first unit does not need the previous result: do it before waiting */
+            float z0[NE];
+            const bool pre = (unit0 < nunits);
+            if (pre) {
+                unit_noise<DT, NW>(g, first, unit0 * EPU, n, z0);
+                /* pin the values here: without this the compiler sinks the arithmetic below the wait */
+#pragma unroll
+                for (int k = 0; k < NE; ++k) asm volatile("" : "+f"(z0[k]));
+            }
             if (threadIdx.x == 0) {
                 bool ok = true;
                 if (!no_ar && t > 1u) {
@@ -439,24 +497,24 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
             }
             __syncthreads();
             if (!s_ok) { alive = false; break; }
-            const Gen g = make_gen(a.w, rank, t);
-            const bool first = (t == 1u);
             const char *prev = no_ar ? a.plain + ((size_t)(p ^ 1u) * P + rank) * a.plain_stride
                                      : a.ring + (size_t)((t + a.ring_len - 2u) % a.ring_len) * a.ring_stride;
             for (uint32_t k = 0; k < a.K; ++k) {
                 const size_t u = unit0 + (size_t)k * kChainThreads;
                 if (u >= nunits) break;
+                uint32_t w[NW];
+                if (k == 0) {
+                    unit_combine<DT, NW>(g, first, prev, u * EPU, n, z0, w);
+                } else {
+                    produce_words<DT, NW>(g, first, prev, u * EPU, n, w);
+                }
                 if (MODE == SIFAR_SPECULATIVE) {
-                    uint32_t w[3];
-                    produce_words<DT, 3>(g, first, prev, u * EPU, n, w);
                     store_slot(reinterpret_cast<uint4 *>(a.slots + ((size_t)p * P + rank) * a.slot_stride), u,
                                w[0], w[1], w[2], e);
                 } else {
-                    uint32_t w[4];
-                    produce_words<DT, 4>(g, first, prev, u * EPU, n, w);
                     const uint32_t bp = (MODE == SIFAR_BARRIER_ONESHOT) ? 0u : p;
                     st_slot(reinterpret_cast<uint4 *>(a.plain + ((size_t)bp * P + rank) * a.plain_stride) + u,
-                            make_uint4(w[0], w[1], w[2], w[3]));
+                            make_uint4(w[0], w[1], w[2], w[NW - 1]));
                 }
             }
             if (MODE == SIFAR_BARRIER_ONESHOT || MODE == SIFAR_DUALBUF) {
@@ -818,6 +876,7 @@ extern "C" int sifar_chain_run(sifar_chain *ch, void *stream)
         a.e0 = no_ar ? ch->base_epoch + ch->runs * (uint32_t)ch->steps : c->h_epoch;
         a.base_epoch = ch->base_epoch; a.steps = (uint32_t)ch->steps;
         a.C = ch->C; a.K = ch->K;
+        a.poll_wide = poll_wide_for(c, ch->n);
         a.bottom_base = ch->runs * (uint32_t)ch->steps * ch->C;
         a.exit_base = ch->runs * (uint32_t)ch->grid;
         a.cs = ch->d_cs; a.chunks = ch->d_chunks; a.stamps = ch->d_stamps; a.retry_steps = ch->d_retry_steps;
