@@ -93,6 +93,19 @@ __device__ __forceinline__ uint32_t atom_add_acq_rel_u32(uint32_t *p, uint32_t v
     return old;
 }
 
+__device__ __forceinline__ uint32_t atom_add_relaxed_u32(uint32_t *p, uint32_t v)
+{
+    uint32_t old;
+    asm volatile("atom.relaxed.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+
+/* Fire-and-forget increment: the issuing thread does not wait for the result. */
+__device__ __forceinline__ void red_add_relaxed_u32(uint32_t *p, uint32_t v)
+{
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+}
+
 __device__ __forceinline__ unsigned long long globaltimer_ns()
 {
     unsigned long long t;

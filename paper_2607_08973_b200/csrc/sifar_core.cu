@@ -65,6 +65,10 @@ struct ReduceArgs {
     uint32_t parity;
     uint32_t check_parity;
     uint32_t poll_wide;      /* speculative: re-load all stale ranks per round (else one at a time) */
+    uint32_t two_phase;      /* 1: deferring regime (see "the reducer kernel")                       */
+    uint32_t janitors;       /* G: how many of the last CTAs sweep up the deferred tiles              */
+    unsigned long long spin_ns;
+    uint32_t *defer;         /* [0] = number of queued tiles, [1..] = their indices */
 };
 
 struct PackArgs {
@@ -86,172 +90,356 @@ constexpr int kThreads = 256;
 /* ------------------------------------------------------------------------ */
 
 /*
- * Completion of a reducer CTA, called by thread 0 after a __syncthreads().  The
- * last CTA re-arms the counter, releases the done flags (bottom barrier, reducer
- * side: every CTA has finished reading) and publishes the new call number.
+ * Completion of a call, by the one thread that knows every CTA is done: statistics,
+ * the done flags of the baseline (bottom barrier, reducer side: every CTA has
+ * finished reading) and the new call number.
  */
 template <int MODE>
-__device__ __forceinline__ void reducer_finish(DevState *st, uint32_t e, int P)
+__device__ __forceinline__ void publish_call(DevState *st, uint32_t e, int P)
 {
-    uint32_t n = gridDim.x;
-    uint32_t arrived = (n > 1) ? atom_add_acq_rel_u32(&st->cta_arrive, 1u) + 1u : 1u;
-    if (arrived == n) {
-        if (n > 1) st_relaxed_u32(&st->cta_arrive, 0u);
-        st->stats[kStatCalls] += 1ull;
-        if (MODE == SIFAR_SPECULATIVE && ld_relaxed_u32(&st->retry_epoch) == e)
-            st->stats[kStatCallsWithRetry] += 1ull;
-        if (MODE == SIFAR_BARRIER_ONESHOT)
-            for (int r = 0; r < P; ++r) st_release_u32(&st->done[r], e);
-        st_release_u32(&st->epoch, e);
-    }
+    atomicAdd(&st->stats[kStatCalls], 1ull);                          /* result unused: fire and forget */
+    if (MODE == SIFAR_SPECULATIVE && ld_relaxed_u32(&st->retry_epoch) == e)
+        atomicAdd(&st->stats[kStatCallsWithRetry], 1ull);
+    if (MODE == SIFAR_BARRIER_ONESHOT)
+        for (int r = 0; r < P; ++r) st_release_u32(&st->done[r], e);
+    /* readers of the call number are ordered after this kernel by the stream or by an event */
+    st_relaxed_u32(&st->epoch, e);
 }
 
 /* ------------------------------------------------------------------------ */
-/* reducer, barrier modes: plain partials behind arrival flags               */
+/* reducer tiles                                                             */
 /* ------------------------------------------------------------------------ */
-template <int DT, int P, int MODE>
-__global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a)
+/*
+ * A tile is kThreads * U consecutive units (16-byte vectors of plain elements,
+ * or slots) and is reduced by one CTA: every thread issues its U * P coalesced
+ * 16-byte loads before the first add.
+ */
+template <int DT, int P>
+__device__ __forceinline__ void tile_plain(const ReduceArgs &a, size_t tile, size_t ntiles)
 {
     constexpr int U = Unroll<P>::value;
     constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;       /* elements per 16-byte vector */
-    DevState *st = a.st;
-    __shared__ uint32_t s_epoch;
-
-    /* Top barrier (Section 3.1, phase 1): warp 0 polls the P arrival flags of this call. */
-    if (threadIdx.x < 32) {
-        const uint2 es = ld_relaxed_u32x2(&st->epoch);
-        const uint32_t e = es.x + 1u;
-        bool ok = (es.y == 0u);
-        if (ok && a.check_parity && (e & 1u) != a.parity) {
-            fail(st, a.host_status, SIFAR_ERR_EPOCH);
-            ok = false;
-        }
-        int polls = 0;
-        if (ok && threadIdx.x < P) {
-            polls = wait_flag_eq(&st->arrive[e & 1u][threadIdx.x], e, a.timeout_ns);
-            if (polls < 0) { fail(st, a.host_status, SIFAR_ERR_TIMEOUT); ok = false; polls = 0; }
-        }
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        polls = __reduce_add_sync(0xFFFFFFFFu, polls);
-        if (threadIdx.x == 0) {
-            s_epoch = ok ? e : 0u;
-            if (polls) atomicAdd(&st->stats[kStatFlagPolls], (unsigned long long)polls);
-        }
-    }
-    __syncthreads();
-    const uint32_t e = s_epoch;
-    if (e == 0u) return;
-
-    /* Pull and reduce (phase 2): P coalesced 16-byte loads per vector, all issued before the first add. */
     const size_t nvec = (size_t)a.n / EPV;
     uint4 *out = reinterpret_cast<uint4 *>(a.out);
-    const size_t stride = (size_t)gridDim.x * kThreads * U;
-    for (size_t base = (size_t)blockIdx.x * kThreads * U + threadIdx.x; base < nvec; base += stride) {
-        uint4 x[U][P];
+    const size_t base = tile * kThreads * U + threadIdx.x;
+    uint4 x[U][P];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t v = base + (size_t)u * kThreads;
-            if (v < nvec) {
+    for (int u = 0; u < U; ++u) {
+        const size_t v = base + (size_t)u * kThreads;
+        if (v < nvec) {
 #pragma unroll
-                for (int r = 0; r < P; ++r) x[u][r] = ld_slot(a.src[r] + v);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t v = base + (size_t)u * kThreads;
-            if (v < nvec) out[v] = sum_vec<DT, P>(x[u], true);
+            for (int r = 0; r < P; ++r) x[u][r] = ld_slot(a.src[r] + v);
         }
     }
-    /* Ragged tail: fewer than EPV elements, one per thread of CTA 0. */
-    const size_t tail0 = nvec * EPV;
-    if (blockIdx.x == 0 && tail0 + threadIdx.x < a.n) {
-        const size_t i = tail0 + threadIdx.x;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const size_t v = base + (size_t)u * kThreads;
+        if (v < nvec) out[v] = sum_vec<DT, P>(x[u], true);
+    }
+    /* Ragged tail (fewer than EPV elements): one element per thread, with the last tile. */
+    const size_t i = nvec * EPV + threadIdx.x;
+    if (tile == ntiles - 1 && i < a.n) {
+        uint32_t w[P];
         if (DT == SIFAR_BF16) {
-            uint32_t w[P];
 #pragma unroll
             for (int r = 0; r < P; ++r)
                 w[r] = ld_relaxed_u16(reinterpret_cast<const uint16_t *>(a.src[r]) + i);
             reinterpret_cast<uint16_t *>(a.out)[i] = (uint16_t)(sum_word<DT, P>(w) & 0xFFFFu);
         } else {
-            uint32_t w[P];
 #pragma unroll
             for (int r = 0; r < P; ++r)
                 w[r] = ld_relaxed_u32(reinterpret_cast<const uint32_t *>(a.src[r]) + i);
             reinterpret_cast<uint32_t *>(a.out)[i] = sum_word<DT, P>(w);
         }
     }
+}
 
-    /* Phase 3 (bottom barrier, baseline only) and publication of the call number. */
+/* Returns false if a slot of this thread was still stale after `limit_ns`. */
+template <int DT, int P>
+__device__ __forceinline__ bool tile_spec(const ReduceArgs &a, size_t tile, size_t nslots, uint32_t e,
+                                          unsigned long long limit_ns, unsigned &reloads)
+{
+    constexpr int U = Unroll<P>::value;
+    const size_t base = tile * kThreads * U + threadIdx.x;
+    bool ok = true;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const size_t s = base + (size_t)u * kThreads;
+        if (s >= nslots || !ok) continue;
+        uint4 x[P];
+#pragma unroll
+        for (int r = 0; r < P; ++r) x[r] = ld_slot(a.src[r] + s);
+        /* validation (Section 4.2): a slot counts iff it carries this call's tag; stale ones are re-loaded */
+        if (!validate_slot<P>(x, a.src, s, e, limit_ns, a.poll_wide != 0u, reloads)) { ok = false; continue; }
+        store_slot_result<DT>(a.out, s, (size_t)a.n, sum_vec<DT, P>(x, false));
+    }
+    return ok;
+}
+
+__host__ __device__ inline size_t tiles_for(size_t units, int per_thread)
+{
+    const size_t per_cta = (size_t)kThreads * per_thread;
+    const size_t t = (units + per_cta - 1) / per_cta;
+    return t ? t : 1;
+}
+
+/* Call number, status and parity check at kernel entry.  Returns 0 if the kernel must not run. */
+__device__ __forceinline__ uint32_t entry_epoch(const ReduceArgs &a, uint2 es)
+{
+    if (es.y != 0u) return 0u;
+    const uint32_t e = es.x + 1u;
+    if (a.check_parity && (e & 1u) != a.parity) {
+        fail(a.st, a.host_status, SIFAR_ERR_EPOCH);
+        return 0u;
+    }
+    return e;
+}
+
+/*
+ * Top barrier (Section 3.1, phase 1) by warp 0: the P arrival flags of this call.
+ * Returns the call number, or 0 with `give_up` telling why: 1 = not arrived
+ * within limit_ns, 2 = error / context dead.
+ */
+template <int P>
+__device__ __forceinline__ uint32_t top_barrier(const ReduceArgs &a, unsigned long long limit_ns, int &give_up)
+{
+    __shared__ uint32_t s_epoch;
+    __shared__ int s_why;
+    DevState *st = a.st;
+    __syncthreads();                                  /* the shared words may still be read from an earlier use */
+    if (threadIdx.x < 32) {
+        const uint2 es = ld_relaxed_u32x2(&st->epoch);
+        const uint32_t e = entry_epoch(a, es);
+        int why = e ? 0 : 2;
+        int polls = 0;
+        if (e && threadIdx.x < P) {
+            polls = wait_flag_eq(&st->arrive[e & 1u][threadIdx.x], e, limit_ns);
+            if (polls < 0) { why = 1; polls = 0; }
+        }
+        why = __reduce_max_sync(0xFFFFFFFFu, why);
+        polls = __reduce_add_sync(0xFFFFFFFFu, polls);
+        if (threadIdx.x == 0) {
+            s_epoch = why ? 0u : e;
+            s_why = why;
+            if (polls) atomicAdd(&st->stats[kStatFlagPolls], (unsigned long long)polls);
+        }
+    }
     __syncthreads();
-    if (threadIdx.x == 0) reducer_finish<MODE>(st, e, P);
+    give_up = s_why;
+    return s_epoch;
 }
 
 /* ------------------------------------------------------------------------ */
-/* reducer, speculative mode: tagged slots, per-slot validation and retry    */
+/* the reducer kernel                                                        */
 /* ------------------------------------------------------------------------ */
+/*
+ * One CTA per tile.  Two regimes, chosen by the host from the grid size:
+ *
+ * in place (grid <= one CTA per SM): a CTA waits for its data as long as the
+ *   time limit allows; it cannot keep the producers off the machine.
+ *
+ * deferring (larger grids): a reducer that fills every SM and then waits would
+ *   keep the very producers it waits for from being scheduled.  So a CTA waits
+ *   only spin_ns; if its tile is still not ready it queues the tile and leaves.
+ *   The G CTAs with the highest indices (G <= one per SM) stay as janitors: they
+ *   wait until everybody has arrived, split the queued tiles among themselves
+ *   and reduce them with the full time limit.  With producers that are on time
+ *   the queue is empty and the janitors cost a short wait at the very end.
+ *
+ * Either way the last CTA out publishes the call (publish_call).
+ */
+struct Roles {
+    uint32_t janitor;      /* 0: leave; k+1: janitor number k                       */
+    uint32_t ndefer;       /* queued tiles (valid for janitors)                     */
+    uint32_t ok;
+};
+
+/* Thread 0 of a CTA in the deferring regime: queue the CTA's tile (made visible before the CTA's arrival). */
+__device__ __forceinline__ void defer_tile(const ReduceArgs &a, size_t tile)
+{
+    const uint32_t slot = atomicAdd(a.defer, 1u);
+    st_relaxed_u32(a.defer + 1u + slot, (uint32_t)tile);
+    __threadfence();
+}
+
+/*
+ * End of a CTA's own tile (all threads call; `alive` = no error seen).  Returns
+ * the CTA's role.
+ *   In place: CTAs count themselves with an atomic whose result they read; the
+ *   last arrival publishes the call.
+ *   Deferring: a CTA's SM slot is worth more than the answer, so it counts itself
+ *   with a fire-and-forget increment and leaves.  The G CTAs with the highest
+ *   indices (dispatched last) are the janitors: they wait until the count is
+ *   complete and then learn how many tiles were queued.
+ * A relaxed count is enough in both regimes: the CTA's loads have returned (its
+ * stores depended on them), which is all the bottom barrier asks; `out` is handed
+ * over by the kernel boundary; a queued tile was fenced by defer_tile().
+ */
+template <int MODE>
+__device__ __forceinline__ Roles cta_arrive(const ReduceArgs &a, uint32_t e, int P, bool alive, bool want_defer,
+                                            size_t tile)
+{
+    __shared__ Roles s_roles;
+    DevState *st = a.st;
+    const uint32_t n = gridDim.x;
+    const bool janitor = a.two_phase && blockIdx.x + a.janitors >= n;
+    /* One barrier: every thread's loads are done.  In place it also collects "somebody saw an error"; in
+       the deferring regime errors are uniform over the CTA and the barrier collects "somebody wants to defer". */
+    int dead;
+    if (a.two_phase) {
+        dead = !alive;
+        if (__syncthreads_or(want_defer) && !dead && threadIdx.x == 0) defer_tile(a, tile);
+    } else {
+        dead = __syncthreads_or(!alive);
+    }
+    if (a.two_phase && !janitor) {
+        if (!dead && threadIdx.x == 0) red_add_relaxed_u32(&st->cta_arrive, 1u);
+        return Roles{0u, 0u, (uint32_t)!dead};
+    }
+    if (threadIdx.x == 0) {
+        Roles r = {0u, 0u, (uint32_t)!dead};
+        if (!dead && !a.two_phase) {
+            const uint32_t arrived = (n > 1u) ? atom_add_relaxed_u32(&st->cta_arrive, 1u) + 1u : 1u;
+            if (arrived == n) {
+                if (n > 1u) st_relaxed_u32(&st->cta_arrive, 0u);
+                publish_call<MODE>(st, e, P);
+            }
+        } else if (!dead) {
+            r.janitor = blockIdx.x + a.janitors - n + 1u;              /* 1 .. G */
+            red_add_relaxed_u32(&st->cta_arrive, 1u);
+            Deadline d;
+            while (ld_acquire_u32(&st->cta_arrive) < n) {
+                if (d.expired(a.timeout_ns)) { fail(st, a.host_status, SIFAR_ERR_TIMEOUT); r.ok = 0u; break; }
+                if ((d.polls % 64u) == 0u && ld_relaxed_u32(&st->status) != 0u) { r.ok = 0u; break; }
+            }
+            r.ndefer = ld_relaxed_u32(a.defer);
+        }
+        s_roles = r;
+    }
+    __syncthreads();
+    return s_roles;
+}
+
+/* Mis-speculation statistics of a CTA: one atomic per warp that re-loaded anything; must precede the arrival. */
+__device__ __forceinline__ void flush_reloads(DevState *st, uint32_t e, unsigned &reloads)
+{
+    const unsigned warp_reloads = __reduce_add_sync(0xFFFFFFFFu, reloads);
+    if (warp_reloads && (threadIdx.x & 31) == 0) {
+        atomicAdd(&st->stats[kStatSlotReloads], (unsigned long long)warp_reloads);
+        if (e) st_relaxed_u32(&st->retry_epoch, e);
+    }
+    reloads = 0;
+}
+
+/* A janitor is done with its share (all threads call).  The last janitor re-arms the counters and publishes. */
+template <int MODE>
+__device__ __forceinline__ void janitor_leave(const ReduceArgs &a, uint32_t e, int P, bool alive)
+{
+    DevState *st = a.st;
+    if (!__syncthreads_and(alive)) return;
+    if (threadIdx.x == 0) {
+        const uint32_t left = atom_add_relaxed_u32(&st->janitor_done, 1u) + 1u;
+        if (left == a.janitors) {
+            st_relaxed_u32(&st->janitor_done, 0u);
+            st_relaxed_u32(&st->cta_arrive, 0u);
+            st_relaxed_u32(a.defer, 0u);
+            publish_call<MODE>(st, e, P);
+        }
+    }
+}
+
+template <int DT, int P, int MODE>
+__global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a)
+{
+    constexpr int U = Unroll<P>::value;
+    constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
+    const size_t ntiles = tiles_for((size_t)a.n / EPV, U);
+    const size_t tile = blockIdx.x;
+    int give_up = 0;
+    uint32_t e = top_barrier<P>(a, a.two_phase ? a.spin_ns : a.timeout_ns, give_up);
+    bool alive = true;
+    if (e == 0u) {
+        if (give_up == 2) return;                                      /* dead context */
+        if (!a.two_phase) {
+            if (threadIdx.x == 0) fail(a.st, a.host_status, SIFAR_ERR_TIMEOUT);
+            return;
+        }
+        /* the ranks are late: queue the tile and free the SM; the call number is still needed to arrive */
+        if (threadIdx.x == 0) defer_tile(a, tile);
+        e = entry_epoch(a, ld_relaxed_u32x2(&a.st->epoch));
+        alive = (e != 0u);
+    } else {
+        tile_plain<DT, P>(a, tile, ntiles);                            /* pull and reduce (phase 2) */
+    }
+    /* phase 3 (bottom barrier, baseline only) and publication of the call number by the last CTA out */
+    const Roles role = cta_arrive<MODE>(a, e, P, alive, false, tile);
+    if (!role.janitor) return;
+    alive = (role.ok != 0u);
+    if (alive && role.ndefer) {
+        alive = (top_barrier<P>(a, a.timeout_ns, give_up) != 0u);
+        if (!alive && give_up == 1 && threadIdx.x == 0) fail(a.st, a.host_status, SIFAR_ERR_TIMEOUT);
+        for (uint32_t i = role.janitor - 1u; i < role.ndefer && alive; i += a.janitors)
+            tile_plain<DT, P>(a, ld_relaxed_u32(a.defer + 1u + i), ntiles);
+    }
+    janitor_leave<MODE>(a, e, P, alive);
+}
+
 template <int DT, int P>
 __global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
 {
     constexpr int U = Unroll<P>::value;
-    constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;       /* elements per slot */
+    constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;
     DevState *st = a.st;
     const size_t nslots = ((size_t)a.n + EPS - 1) / EPS;
-
-    /* The call number is loaded together with the first slots: no dependent round trip before the data. */
-    const uint2 es = ld_relaxed_u32x2(&st->epoch);
-    uint32_t e = 0;
-    bool alive = true;
+    const size_t tile = blockIdx.x;
+    const unsigned long long limit_ns = a.two_phase ? a.spin_ns : a.timeout_ns;
     unsigned reloads = 0;
 
-    const size_t stride = (size_t)gridDim.x * kThreads * U;
-    for (size_t base = (size_t)blockIdx.x * kThreads * U + threadIdx.x; base < nslots && alive; base += stride) {
-        uint4 x[U][P];
+    /* The call number is loaded together with the slots (no dependent round trip before the data), by one
+       thread per CTA: a word that every warp of a large grid loads becomes a hot spot in its L2 slice. */
+    __shared__ uint2 s_es;
+    if (threadIdx.x == 0) s_es = ld_relaxed_u32x2(&st->epoch);
+    const size_t base = tile * kThreads * U + threadIdx.x;
+    uint4 x[U][P];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const size_t s = base + (size_t)u * kThreads;
+        if (s < nslots) {
+#pragma unroll
+            for (int r = 0; r < P; ++r) x[u][r] = ld_slot(a.src[r] + s);
+        }
+    }
+    __syncthreads();
+    const uint32_t e = entry_epoch(a, s_es);
+    bool alive = (e != 0u);
+    bool ok = true;
+    if (alive) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const size_t s = base + (size_t)u * kThreads;
-            if (s < nslots) {
-#pragma unroll
-                for (int r = 0; r < P; ++r) x[u][r] = ld_slot(a.src[r] + s);
-            }
-        }
-        if (e == 0u) {
-            e = es.x + 1u;
-            if (es.y != 0u) { alive = false; break; }
-            if (a.check_parity && (e & 1u) != a.parity) {
-                fail(st, a.host_status, SIFAR_ERR_EPOCH);
-                alive = false;
-                break;
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t s = base + (size_t)u * kThreads;
-            if (s >= nslots) continue;
-            if (!validate_slot<P>(x[u], a.src, s, e, a.timeout_ns, a.poll_wide != 0u, reloads)) {
-                fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
-                alive = false;
-                break;
-            }
+            if (s >= nslots || !ok) continue;
+            /* validation (Section 4.2): a slot counts iff it carries this call's tag; stale ones are re-loaded */
+            if (!validate_slot<P>(x[u], a.src, s, e, limit_ns, a.poll_wide != 0u, reloads)) { ok = false; continue; }
             store_slot_result<DT>(a.out, s, (size_t)a.n, sum_vec<DT, P>(x[u], false));
         }
+        if (!a.two_phase && !ok) {
+            fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+            alive = false;
+        }
     }
-
-    /* Threads without a slot still need the call number for the completion step. */
-    if (e == 0u && alive) {
-        e = es.x + 1u;
-        if (es.y != 0u) alive = false;
-        else if (a.check_parity && (e & 1u) != a.parity) { fail(st, a.host_status, SIFAR_ERR_EPOCH); alive = false; }
+    flush_reloads(st, e, reloads);
+    /* deferring regime: a slot that stayed stale past the short limit sends the whole tile to a janitor */
+    const Roles role = cta_arrive<SIFAR_SPECULATIVE>(a, e, P, alive, a.two_phase && !ok, tile);
+    if (!role.janitor) return;
+    alive = (role.ok != 0u);
+    for (uint32_t i = role.janitor - 1u; i < role.ndefer && alive; i += a.janitors) {
+        if (!tile_spec<DT, P>(a, ld_relaxed_u32(a.defer + 1u + i), nslots, e, a.timeout_ns, reloads)) {
+            fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+            alive = false;
+        }
     }
-
-    /* Mis-speculation statistics: one atomic per warp that re-loaded anything. */
-    const unsigned warp_reloads = __reduce_add_sync(0xFFFFFFFFu, reloads);
-    if (warp_reloads && (threadIdx.x & 31) == 0) {
-        atomicAdd(&st->stats[kStatSlotReloads], (unsigned long long)warp_reloads);
-        st_relaxed_u32(&st->retry_epoch, e);
-    }
-    const int all_alive = __syncthreads_and(alive);
-    if (!all_alive) return;
-    if (threadIdx.x == 0) reducer_finish<SIFAR_SPECULATIVE>(st, e, P);
+    flush_reloads(st, e, reloads);
+    janitor_leave<SIFAR_SPECULATIVE>(a, e, P, alive);
 }
 
 /* ------------------------------------------------------------------------ */
@@ -358,16 +546,6 @@ __global__ void k_set_epoch(DevState *st, uint32_t e) { st->epoch = e; }
 /* ------------------------------------------------------------------------ */
 /* launch geometry                                                           */
 /* ------------------------------------------------------------------------ */
-static int reduce_grid(const sifar_ctx *ctx, size_t units, int per_thread)
-{
-    const size_t per_cta = (size_t)kThreads * per_thread;
-    size_t ctas = (units + per_cta - 1) / per_cta;
-    const size_t cap = (size_t)ctx->sm_count * 4;          /* 4 CTAs of 256 threads per SM: one wave */
-    if (ctas > cap) ctas = cap;
-    if (ctas < 1) ctas = 1;
-    return (int)ctas;
-}
-
 template <int DT, int P>
 static cudaError_t launch_reduce_p(int mode, int grid, cudaStream_t s, const ReduceArgs &a)
 {
@@ -402,9 +580,17 @@ uint32_t sifar::poll_wide_for(const sifar_ctx *ctx, size_t n)
     return slots_for(ctx->dtype, n) * (size_t)ctx->P <= ctx->poll_wide_max ? 1u : 0u;
 }
 
-namespace sifar {
-
 static int unroll_for(int P) { return P <= 2 ? 4 : P <= 4 ? 2 : 1; }
+
+static size_t reduce_units(const sifar_ctx *ctx, size_t n, int mode)
+{
+    return mode == SIFAR_SPECULATIVE ? sifar::slots_for(ctx->dtype, n) : n * sifar::elem_size(ctx->dtype) / 16;
+}
+
+/* Kernels one all-reduce call launches. */
+int sifar::reduce_launch_count(const sifar_ctx *, size_t, int) { return 1; }
+
+namespace sifar {
 
 int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
 {
@@ -424,12 +610,16 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
     a.parity = rl.parity;
     a.check_parity = (rl.mode != SIFAR_BARRIER_ONESHOT);
     a.poll_wide = poll_wide_for(ctx, rl.n);
-    size_t units = (rl.mode == SIFAR_SPECULATIVE) ? slots_for(ctx->dtype, rl.n)
-                                                  : (rl.n * elem_size(ctx->dtype) + 15) / 16;
-    const int grid = reduce_grid(ctx, units, unroll_for(ctx->P));
+    a.defer = ctx->d_defer;
+    a.spin_ns = ctx->spin_ns < ctx->timeout_ns ? ctx->spin_ns : ctx->timeout_ns;
+    /* One tile per CTA.  Up to one CTA per SM the reducer cannot crowd out the producers and waits in
+       place; beyond that it runs at full occupancy, waits briefly, and its last CTAs sweep up. */
+    const size_t ntiles = tiles_for(reduce_units(ctx, rl.n, rl.mode), unroll_for(ctx->P));
+    a.two_phase = ntiles > (size_t)ctx->sm_count ? 1u : 0u;
+    a.janitors = (uint32_t)ctx->sm_count;
     cudaError_t err = (ctx->dtype == SIFAR_BF16)
-        ? launch_reduce_dt<SIFAR_BF16>(ctx->P, rl.mode, grid, stream, a)
-        : launch_reduce_dt<SIFAR_F32>(ctx->P, rl.mode, grid, stream, a);
+        ? launch_reduce_dt<SIFAR_BF16>(ctx->P, rl.mode, (int)ntiles, stream, a)
+        : launch_reduce_dt<SIFAR_F32>(ctx->P, rl.mode, (int)ntiles, stream, a);
     SIFAR_CUDA(err);
     return SIFAR_OK;
 }
@@ -491,6 +681,8 @@ extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
     c->P = P; c->dtype = dtype; c->max_elems = max_elems;
     c->timeout_ns = 200000ull * 1000ull;
     c->poll_wide_max = 16384;
+    c->spin_ns = 5000;
+    if (const char *env = getenv("SIFAR_SPIN_NS")) c->spin_ns = strtoull(env, nullptr, 10);
     if (const char *env = getenv("SIFAR_POLL_WIDE_MAX")) c->poll_wide_max = (size_t)strtoull(env, nullptr, 10);
     cudaError_t e = cudaGetDevice(&c->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
@@ -500,6 +692,9 @@ extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
     if (e == cudaSuccess) e = cudaMalloc(&c->d_plain, plain_bytes);
     if (e == cudaSuccess) e = cudaMalloc(&c->d_slots, slot_bytes);
     if (e == cudaSuccess) e = cudaMalloc(&c->d_state, sizeof(DevState));
+    const size_t defer_words = 2 + (slots_for(dtype, max_elems) + kThreads - 1) / kThreads;
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_defer, defer_words * sizeof(uint32_t));
+    if (e == cudaSuccess) e = cudaMemset(c->d_defer, 0, defer_words * sizeof(uint32_t));
     if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->h_status, sizeof(int), cudaHostAllocMapped);
     if (e == cudaSuccess) { *c->h_status = 0; e = cudaHostGetDevicePointer((void **)&c->d_status_alias, (void *)c->h_status, 0); }
     if (e == cudaSuccess) e = cudaMemset(c->d_plain, 0, plain_bytes);
@@ -514,6 +709,7 @@ extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
         if (c->d_plain) cudaFree(c->d_plain);
         if (c->d_slots) cudaFree(c->d_slots);
         if (c->d_state) cudaFree(c->d_state);
+        if (c->d_defer) cudaFree(c->d_defer);
         if (c->h_status) cudaFreeHost((void *)c->h_status);
         if (c->host_stream) cudaStreamDestroy(c->host_stream);
         delete c;
@@ -531,6 +727,7 @@ extern "C" int sifar_destroy(sifar_ctx *c)
     cudaFree(c->d_plain);
     cudaFree(c->d_slots);
     cudaFree(c->d_state);
+    cudaFree(c->d_defer);
     if (c->d_stage_in) cudaFree(c->d_stage_in);
     if (c->d_stage_out) cudaFree(c->d_stage_out);
     cudaFreeHost((void *)c->h_status);
@@ -729,6 +926,7 @@ extern "C" int sifar_reset(sifar_ctx *c, void *stream)
     SIFAR_CUDA(cudaDeviceSynchronize());
     SIFAR_CUDA(cudaMemsetAsync(c->d_slots, 0, c->slot_stride * 2 * c->P, s));
     SIFAR_CUDA(cudaMemsetAsync(c->d_state, 0, sizeof(DevState), s));
+    SIFAR_CUDA(cudaMemsetAsync(c->d_defer, 0, sizeof(uint32_t), s));
     SIFAR_CUDA(cudaStreamSynchronize(s));
     *c->h_status = 0;
     c->h_epoch = 0;

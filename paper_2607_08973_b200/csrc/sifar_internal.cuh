@@ -29,7 +29,8 @@ struct __align__(128) DevState {
     /* line 1: last-CTA detection of the reducer; retry marker */
     uint32_t cta_arrive;
     uint32_t retry_epoch;            /* call number of the last call that re-loaded a slot       */
-    uint32_t pad1[30];
+    uint32_t janitor_done;           /* janitor CTAs that have finished their share              */
+    uint32_t pad1[29];
     /* lines 2-3: arrival flags, one 128-byte line per parity (top barrier) */
     uint32_t arrive[2][32];
     /* line 4: done flags (bottom barrier, BARRIER_ONESHOT) */
@@ -76,11 +77,13 @@ struct sifar_ctx {
     char *d_plain;                   /* [parity][rank] plain buffers                     */
     char *d_slots;                   /* [parity][rank] slot buffers                      */
     sifar::DevState *d_state;
+    uint32_t *d_defer;               /* queued tiles of the deferring reducer: count, then tile indices */
     volatile int *h_status;          /* pinned, mapped                                   */
     int *d_status_alias;             /* device alias of h_status                         */
     uint32_t h_epoch;                /* calls enqueued so far                            */
     uint32_t last_mode0_epoch;       /* last BARRIER_ONESHOT call (0: none): whose done flags a producer waits for */
     unsigned long long timeout_ns;
+    unsigned long long spin_ns;      /* deferring reducer: how long a CTA waits before it queues its tile     */
     size_t poll_wide_max;            /* speculative: wide polling up to this many (slot, rank) pairs per call */
     /* staging for sifar_allreduce_host, allocated on first use */
     char *d_stage_in;
@@ -115,6 +118,7 @@ struct ReduceLaunch {
 
 int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream);
 uint32_t poll_wide_for(const sifar_ctx *ctx, size_t n);
+int reduce_launch_count(const sifar_ctx *ctx, size_t n, int mode);
 
 }  /* namespace sifar */
 #endif

@@ -15,19 +15,17 @@ namespace sifar {
 /* ------------------------------------------------------------------------ */
 
 /*
- * Reading %globaltimer is slow next to an L2 round trip, so the time limit is
- * only looked at every kPollsPerClockCheck failed polls; a poll costs at least
- * one trip to the L2, which keeps the overshoot to a few tens of microseconds.
+ * Time limit of a polling loop.  %globaltimer costs a handful of cycles next to
+ * the L2 round trip of the poll itself, so it is read after every failed poll;
+ * the clock starts at the first failed poll.
  */
-constexpr unsigned kPollsPerClockCheck = 64;
-
 struct Deadline {
     unsigned long long t0 = 0;
     unsigned polls = 0;
     /* Call after a failed poll; true once the limit has passed. */
     __device__ __forceinline__ bool expired(unsigned long long timeout_ns)
     {
-        if ((++polls % kPollsPerClockCheck) != 0u) return false;
+        ++polls;
         const unsigned long long now = globaltimer_ns();
         if (t0 == 0) { t0 = now; return false; }
         return now - t0 > timeout_ns;

@@ -375,7 +375,7 @@ __device__ __forceinline__ bool chain_wait(const uint32_t *flag, uint32_t want, 
         const uint32_t v = ld_acquire_u32(flag);
         if (GE ? (v >= want) : (v == want)) return true;
         if (d.expired(timeout_ns)) { fail(st, host_status, SIFAR_ERR_TIMEOUT); return false; }
-        if ((d.polls % kPollsPerClockCheck) == 0u && ld_relaxed_u32(&st->status) != 0u) return false;
+        if ((d.polls % 64u) == 0u && ld_relaxed_u32(&st->status) != 0u) return false;
     }
 }
 
@@ -818,7 +818,7 @@ extern "C" sifar_chain *sifar_chain_create(sifar_ctx *c, const sifar_workload *w
         for (int r = 0; r <= c->P; ++r) SIFAR_CUDA(cudaEventCreateWithFlags(&ch->ev_join[r], cudaEventDisableTiming));
         ch->ev_step.assign((size_t)ch->steps, nullptr);
         for (int s = 0; s < ch->steps; ++s) SIFAR_CUDA(cudaEventCreateWithFlags(&ch->ev_step[s], cudaEventDisableTiming));
-        ch->launches_per_run = ch->steps * (c->P + (mode == kModeNoAllreduce ? 0 : 1));
+        ch->launches_per_run = ch->steps * (c->P + (mode == kModeNoAllreduce ? 0 : reduce_launch_count(c, n, mode)));
         if (impl == SIFAR_CHAIN_GRAPH) {
             /* capture one run; every later replay finds the same parities because steps_per_run is even */
             cudaStream_t cap;
