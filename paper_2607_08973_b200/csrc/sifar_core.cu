@@ -64,7 +64,7 @@ struct ReduceArgs {
     unsigned long long timeout_ns;
     uint32_t parity;
     uint32_t check_parity;
-    uint32_t poll_wide;      /* speculative: re-load all stale ranks per round (else one at a time) */
+    PollShape poll;          /* speculative: how stale slots are re-polled (see validate_slot)        */
     uint32_t two_phase;      /* 1: deferring regime (see "the reducer kernel")                       */
     uint32_t janitors;       /* G: how many of the last CTAs sweep up the deferred tiles              */
     unsigned long long spin_ns;
@@ -170,7 +170,7 @@ __device__ __forceinline__ bool tile_spec(const ReduceArgs &a, size_t tile, size
 #pragma unroll
         for (int r = 0; r < P; ++r) x[r] = ld_slot(a.src[r] + s);
         /* validation (Section 4.2): a slot counts iff it carries this call's tag; stale ones are re-loaded */
-        if (!validate_slot<P>(x, a.src, s, e, limit_ns, a.poll_wide != 0u, reloads)) { ok = false; continue; }
+        if (!validate_slot<P>(x, a.src, s, e, limit_ns, a.poll, reloads)) { ok = false; continue; }
         store_slot_result<DT>(a.out, s, (size_t)a.n, sum_vec<DT, P>(x, false));
     }
     return ok;
@@ -419,7 +419,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
             const size_t s = base + (size_t)u * kThreads;
             if (s >= nslots || !ok) continue;
             /* validation (Section 4.2): a slot counts iff it carries this call's tag; stale ones are re-loaded */
-            if (!validate_slot<P>(x[u], a.src, s, e, limit_ns, a.poll_wide != 0u, reloads)) { ok = false; continue; }
+            if (!validate_slot<P>(x[u], a.src, s, e, limit_ns, a.poll, reloads)) { ok = false; continue; }
             store_slot_result<DT>(a.out, s, (size_t)a.n, sum_vec<DT, P>(x[u], false));
         }
         if (!a.two_phase && !ok) {
@@ -574,10 +574,14 @@ static cudaError_t launch_reduce_dt(int P, int mode, int grid, cudaStream_t s, c
 
 }  /* namespace sifar */
 
-/* Wide polling while the whole grid's polling volume per round stays small (see validate_slot). */
-uint32_t sifar::poll_wide_for(const sifar_ctx *ctx, size_t n)
+/* Polling shape from the number of (slot, rank) pairs a waiting grid re-polls per round (see validate_slot). */
+sifar::PollShape sifar::poll_shape_for(const sifar_ctx *ctx, size_t n)
 {
-    return slots_for(ctx->dtype, n) * (size_t)ctx->P <= ctx->poll_wide_max ? 1u : 0u;
+    const size_t pairs = slots_for(ctx->dtype, n) * (size_t)ctx->P;
+    PollShape p;
+    p.wide = pairs <= ctx->poll_wide_max ? 1u : 0u;
+    p.pace_ns = pairs <= ctx->poll_pace_min ? 0u : ctx->poll_pace_ns;
+    return p;
 }
 
 static int unroll_for(int P) { return P <= 2 ? 4 : P <= 4 ? 2 : 1; }
@@ -585,6 +589,11 @@ static int unroll_for(int P) { return P <= 2 ? 4 : P <= 4 ? 2 : 1; }
 static size_t reduce_units(const sifar_ctx *ctx, size_t n, int mode)
 {
     return mode == SIFAR_SPECULATIVE ? sifar::slots_for(ctx->dtype, n) : n * sifar::elem_size(ctx->dtype) / 16;
+}
+
+size_t sifar::reduce_tiles(const sifar_ctx *ctx, size_t n, int mode)
+{
+    return tiles_for(reduce_units(ctx, n, mode), unroll_for(ctx->P));
 }
 
 /* Kernels one all-reduce call launches. */
@@ -609,7 +618,7 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
     a.timeout_ns = ctx->timeout_ns;
     a.parity = rl.parity;
     a.check_parity = (rl.mode != SIFAR_BARRIER_ONESHOT);
-    a.poll_wide = poll_wide_for(ctx, rl.n);
+    a.poll = poll_shape_for(ctx, rl.n);
     a.defer = ctx->d_defer;
     a.spin_ns = ctx->spin_ns < ctx->timeout_ns ? ctx->spin_ns : ctx->timeout_ns;
     /* One tile per CTA.  Up to one CTA per SM the reducer cannot crowd out the producers and waits in
@@ -683,7 +692,11 @@ extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
     c->poll_wide_max = 16384;
     c->spin_ns = 5000;
     if (const char *env = getenv("SIFAR_SPIN_NS")) c->spin_ns = strtoull(env, nullptr, 10);
+    c->poll_pace_min = 16384;
+    c->poll_pace_ns = 0;
     if (const char *env = getenv("SIFAR_POLL_WIDE_MAX")) c->poll_wide_max = (size_t)strtoull(env, nullptr, 10);
+    if (const char *env = getenv("SIFAR_POLL_PACE_MIN")) c->poll_pace_min = (size_t)strtoull(env, nullptr, 10);
+    if (const char *env = getenv("SIFAR_POLL_PACE_NS")) c->poll_pace_ns = (uint32_t)strtoul(env, nullptr, 10);
     cudaError_t e = cudaGetDevice(&c->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
     c->plain_stride = round_up(max_elems * elem_size(dtype), 256);

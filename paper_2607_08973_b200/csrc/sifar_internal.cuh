@@ -85,6 +85,8 @@ struct sifar_ctx {
     unsigned long long timeout_ns;
     unsigned long long spin_ns;      /* deferring reducer: how long a CTA waits before it queues its tile     */
     size_t poll_wide_max;            /* speculative: wide polling up to this many (slot, rank) pairs per call */
+    size_t poll_pace_min;            /* ... paced polling above this many pairs                              */
+    uint32_t poll_pace_ns;
     /* staging for sifar_allreduce_host, allocated on first use */
     char *d_stage_in;
     char *d_stage_out;
@@ -117,8 +119,10 @@ struct ReduceLaunch {
 };
 
 int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream);
-uint32_t poll_wide_for(const sifar_ctx *ctx, size_t n);
+struct PollShape;
+PollShape poll_shape_for(const sifar_ctx *ctx, size_t n);
 int reduce_launch_count(const sifar_ctx *ctx, size_t n, int mode);
+size_t reduce_tiles(const sifar_ctx *ctx, size_t n, int mode);     /* CTAs of the reducer kernel for n elements */
 
 }  /* namespace sifar */
 #endif

@@ -15,17 +15,20 @@ namespace sifar {
 /* ------------------------------------------------------------------------ */
 
 /*
- * Time limit of a polling loop.  %globaltimer costs a handful of cycles next to
- * the L2 round trip of the poll itself, so it is read after every failed poll;
- * the clock starts at the first failed poll.
+ * Time limit of a polling loop.  The clock (%globaltimer) is read on every
+ * kPollsPerClockCheck-th failed poll only: reading it on every poll measurably
+ * slows the poll loops of the persistent chain.  A poll costs at least one L2
+ * round trip (~0.3 us), so a limit is overshot by a few microseconds at most.
  */
+constexpr unsigned kPollsPerClockCheck = 8;
+
 struct Deadline {
     unsigned long long t0 = 0;
     unsigned polls = 0;
     /* Call after a failed poll; true once the limit has passed. */
     __device__ __forceinline__ bool expired(unsigned long long timeout_ns)
     {
-        ++polls;
+        if ((++polls % kPollsPerClockCheck) != 1u) return false;
         const unsigned long long now = globaltimer_ns();
         if (t0 == 0) { t0 = now; return false; }
         return now - t0 > timeout_ns;
@@ -99,26 +102,26 @@ template <int P> struct Unroll { static constexpr int value = (P <= 2) ? 4 : (P 
  * every tag matches or the time limit passes.  Returns false on time-out.
  * `reloads` counts the extra loads.
  *
- * Two polling shapes.  wide: every stale rank is re-loaded each round; the last
- * arrival is seen one L2 round trip later, at P loads per waiting thread and
- * round.  narrow: only the lowest stale rank is polled; when it turns valid one
- * wide round follows.  Narrow costs one more round trip after the last arrival
- * but keeps the polling traffic of a large waiting grid from starving the
- * producers' stores of L2 bandwidth.
+ * Polling shapes (WIDE, pace_ns):
+ *   wide    every stale rank is re-loaded each round: the last arrival is seen one
+ *           L2 round trip later, at up to P loads per waiting thread and round.
+ *   narrow  only the lowest stale rank is polled; when it turns valid one wide
+ *           round follows.  One more round trip after the last arrival, 1/P of
+ *           the polling traffic.
+ *   pace_ns sleep between rounds.
+ * A large waiting grid that polls wide and unpaced takes L2 bandwidth away from
+ * the very producers it waits for; the host picks the shape from the grid size.
  */
-template <int P>
-__device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const *src, size_t s, uint32_t e,
-                                              unsigned long long timeout_ns, bool wide, unsigned &reloads)
+template <int P, bool WIDE>
+__device__ __forceinline__ bool revalidate(uint4 (&x)[P], uint32_t stale, const uint4 *const *src, size_t s,
+                                           uint32_t e, unsigned long long timeout_ns, uint32_t pace_ns,
+                                           unsigned &reloads)
 {
-    uint32_t stale = 0;
-#pragma unroll
-    for (int r = 0; r < P; ++r) stale |= (uint32_t)(x[r].w != e) << r;
-    if (stale == 0u) return true;
     Deadline d;
-    bool burst = wide;
+    bool burst = WIDE;
     do {
         /* issue every pending load before looking at any result, so that the re-loads overlap */
-        const uint32_t pending = burst ? stale : (stale & (0u - stale));
+        const uint32_t pending = (WIDE || burst) ? stale : (stale & (0u - stale));
 #pragma unroll
         for (int r = 0; r < P; ++r)
             if (pending & (1u << r)) x[r] = ld_slot(src[r] + s);
@@ -127,10 +130,30 @@ __device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const 
         for (int r = 0; r < P; ++r)
             if ((pending & (1u << r)) && x[r].w == e) stale &= ~(1u << r);
         reloads += __popc(pending);
-        burst = wide || (!burst && stale != before);     /* narrow: the polled rank arrived, look at all others once */
-        if (stale && d.expired(timeout_ns)) return false;
+        if (!WIDE) burst = !burst && stale != before;    /* the polled rank arrived: look at all others once */
+        if (stale) {
+            if (d.expired(timeout_ns)) return false;
+            if (pace_ns) __nanosleep(pace_ns);
+        }
     } while (stale);
     return true;
+}
+
+struct PollShape {
+    uint32_t wide;
+    uint32_t pace_ns;
+};
+
+template <int P>
+__device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const *src, size_t s, uint32_t e,
+                                              unsigned long long timeout_ns, PollShape shape, unsigned &reloads)
+{
+    uint32_t stale = 0;
+#pragma unroll
+    for (int r = 0; r < P; ++r) stale |= (uint32_t)(x[r].w != e) << r;
+    if (stale == 0u) return true;
+    return shape.wide ? revalidate<P, true>(x, stale, src, s, e, timeout_ns, shape.pace_ns, reloads)
+                      : revalidate<P, false>(x, stale, src, s, e, timeout_ns, shape.pace_ns, reloads);
 }
 
 /* ------------------------------------------------------------------------ */

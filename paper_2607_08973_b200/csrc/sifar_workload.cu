@@ -18,6 +18,7 @@
  * ordering (identical in all modes) and every arrow is one dependent trip
  * through the L2.
  */
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -221,6 +222,7 @@ __device__ __forceinline__ void spin_ns(uint32_t ns)
 
 constexpr int kModeNoAllreduce = SIFAR_CHAIN_NO_ALLREDUCE;
 constexpr unsigned kMaxDelayNs = 1000000u;       /* producer delays are capped at 1 ms */
+constexpr size_t kConcurrentTiles = 48;          /* see sifar_chain::concurrent */
 
 /* ------------------------------------------------------------------------ */
 /* producer kernel of the stream / graph chains                              */
@@ -356,7 +358,7 @@ struct PersistArgs {
     uint32_t C;                     /* chunks = reducer CTAs               */
     uint32_t K;                     /* units per thread and step           */
     uint32_t bottom_base, exit_base;
-    uint32_t poll_wide;
+    PollShape poll;
     ChainDev *cs;
     ChunkFlags *chunks;
     unsigned long long *stamps;     /* steps + 1                           */
@@ -441,7 +443,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                 for (int r = 0; r < P; ++r) x[r] = ld_slot(src[r] + u);
                 if (MODE == SIFAR_SPECULATIVE) {
                     const unsigned before = reloads;
-                    if (!validate_slot<P>(x, src, u, e, a.timeout_ns, a.poll_wide != 0u, reloads)) {
+                    if (!validate_slot<P>(x, src, u, e, a.timeout_ns, a.poll, reloads)) {
                         fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
                         alive = false;
                         break;
@@ -604,6 +606,17 @@ struct sifar_chain {
     cudaStream_t red;
     cudaEvent_t ev_fork;
     cudaEvent_t ev_join[kMaxRanks + 1];
+    cudaEvent_t ev_prod[kMaxRanks];
+    /*
+     * Stream / graph chains: may the reducer kernel of a step start without waiting for that step's
+     * producers?  CUDA does not promise that independently launched kernels run at the same time, and on
+     * B200 the producers of a graph step were measured to run only on SMs that hold no CTA of an
+     * already polling speculative reducer (step time ~ 1 / free SMs, no progress at one CTA per SM).
+     * Up to kConcurrentTiles reducer CTAs the step is left unordered, which is what the speculative and
+     * barrier protocols are about at decode payloads; above it the reducer is ordered behind the
+     * producers by events: there the transfer dominates and the early start buys nothing.
+     */
+    bool concurrent;
     std::vector<cudaEvent_t> ev_step;
     cudaGraph_t graph;
     cudaGraphExec_t exec;
@@ -659,7 +672,8 @@ static int enqueue_run(sifar_chain *ch, cudaStream_t origin, uint32_t first_t)
     const size_t units = (ch->mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, ch->n)
                                                          : (ch->n * elem_size(c->dtype) + 15) / 16;
     size_t pgrid = (units + kProdThreads - 1) / kProdThreads;
-    const size_t cap = (size_t)c->sm_count * 2;
+    size_t cap = (size_t)c->sm_count * 2;
+    if (const char *env = getenv("SIFAR_PROD_CAP")) cap = (size_t)atoi(env);
     if (pgrid > cap) pgrid = cap;
 
     for (int s = 0; s < ch->steps; ++s) {
@@ -680,6 +694,11 @@ static int enqueue_run(sifar_chain *ch, cudaStream_t origin, uint32_t first_t)
                 ? launch_produce_dt<SIFAR_BF16>(ch->mode, (int)pgrid, ch->prod[r], a)
                 : launch_produce_dt<SIFAR_F32>(ch->mode, (int)pgrid, ch->prod[r], a);
             SIFAR_CUDA(err);
+            if (!no_ar && !ch->concurrent) {
+                /* large reducer grid: order it behind the producers (see sifar_chain::concurrent) */
+                SIFAR_CUDA(cudaEventRecord(ch->ev_prod[r], ch->prod[r]));
+                SIFAR_CUDA(cudaStreamWaitEvent(ch->red, ch->ev_prod[r], 0));
+            }
         }
         if (!no_ar) {
             ReduceLaunch rl;
@@ -742,6 +761,7 @@ static void chain_free(sifar_chain *ch)
     if (ch->red) cudaStreamDestroy(ch->red);
     if (ch->ev_fork) cudaEventDestroy(ch->ev_fork);
     for (int r = 0; r <= kMaxRanks; ++r) if (ch->ev_join[r]) cudaEventDestroy(ch->ev_join[r]);
+    for (int r = 0; r < kMaxRanks; ++r) if (ch->ev_prod[r]) cudaEventDestroy(ch->ev_prod[r]);
     for (cudaEvent_t e : ch->ev_step) if (e) cudaEventDestroy(e);
     if (ch->exec) cudaGraphExecDestroy(ch->exec);
     if (ch->graph) cudaGraphDestroy(ch->graph);
@@ -816,6 +836,8 @@ extern "C" sifar_chain *sifar_chain_create(sifar_ctx *c, const sifar_workload *w
         SIFAR_CUDA(cudaStreamCreateWithFlags(&ch->red, cudaStreamNonBlocking));
         SIFAR_CUDA(cudaEventCreateWithFlags(&ch->ev_fork, cudaEventDisableTiming));
         for (int r = 0; r <= c->P; ++r) SIFAR_CUDA(cudaEventCreateWithFlags(&ch->ev_join[r], cudaEventDisableTiming));
+        for (int r = 0; r < c->P; ++r) SIFAR_CUDA(cudaEventCreateWithFlags(&ch->ev_prod[r], cudaEventDisableTiming));
+        ch->concurrent = reduce_tiles(c, n, mode == kModeNoAllreduce ? SIFAR_DUALBUF : mode) <= kConcurrentTiles;
         ch->ev_step.assign((size_t)ch->steps, nullptr);
         for (int s = 0; s < ch->steps; ++s) SIFAR_CUDA(cudaEventCreateWithFlags(&ch->ev_step[s], cudaEventDisableTiming));
         ch->launches_per_run = ch->steps * (c->P + (mode == kModeNoAllreduce ? 0 : reduce_launch_count(c, n, mode)));
@@ -876,7 +898,7 @@ extern "C" int sifar_chain_run(sifar_chain *ch, void *stream)
         a.e0 = no_ar ? ch->base_epoch + ch->runs * (uint32_t)ch->steps : c->h_epoch;
         a.base_epoch = ch->base_epoch; a.steps = (uint32_t)ch->steps;
         a.C = ch->C; a.K = ch->K;
-        a.poll_wide = poll_wide_for(c, ch->n);
+        a.poll = poll_shape_for(c, ch->n);
         a.bottom_base = ch->runs * (uint32_t)ch->steps * ch->C;
         a.exit_base = ch->runs * (uint32_t)ch->grid;
         a.cs = ch->d_cs; a.chunks = ch->d_chunks; a.stamps = ch->d_stamps; a.retry_steps = ch->d_retry_steps;
