@@ -170,6 +170,38 @@ int sifar_reset(sifar_ctx *ctx, void *stream);
  */
 int sifar_debug_set_epoch(sifar_ctx *ctx, unsigned calls_so_far);
 
+/*
+ * All-reduce without any allocation.  The paper has no counterpart for this call.
+ *
+ * For callers that must not allocate device memory: an engine that gave the whole
+ * device to its own arena at start-up and may not call cudaMalloc afterwards, or
+ * a latency-critical loop that cannot afford the device-wide synchronization an
+ * allocation implies.  It reduces P caller-owned plain partials that are already
+ * complete in the order of `stream` (no flags, no tags, no context) into `out`:
+ * same arithmetic as sifar_allreduce().
+ *
+ *   rank_ptrs  host array of P device pointers (1 <= P <= 8), n plain elements each,
+ *              16-byte aligned, read only.
+ *   out        device, n plain elements, 16-byte aligned, must not overlap an input.
+ *   n          at most sifar_noalloc_max_elems() = 2^20 elements per rank; larger n
+ *              is refused with SIFAR_ERR_INVALID (use a context instead).  n = 0 is
+ *              a no-op.
+ *
+ * The kernel's bookkeeping (the count of finished CTAs by which the last CTA
+ * knows it is last, and two call counters; 256 bytes) lives in a fixed array in
+ * the library's device image: every GPU that loads the library holds it until
+ * the process exits.  The first call on a device looks up the array's device
+ * address (cudaGetSymbolAddress, with that device current) and caches it; make
+ * that first call before any stream capture begins.  The call itself enqueues a
+ * 4-byte clear of the CTA count and one kernel on `stream`; it calls no
+ * cudaMalloc, cudaFree or other allocating routine and does not synchronize.
+ * All calls on a device share the array, which keeps the previous call's
+ * counters: calls that overlap in time on the GPU (different streams without an
+ * ordering between them) race on it and are not supported.
+ */
+int sifar_allreduce_noalloc(const void *const *rank_ptrs, int P, void *out, size_t n, int dtype, void *stream);
+size_t sifar_noalloc_max_elems(void);
+
 /* Geometry helpers (no device work). */
 size_t sifar_slot_count(int dtype, size_t n);          /* slots needed for n elements  */
 size_t sifar_algorithmic_bytes(int P, int dtype, size_t n, int mode);  /* bytes the method must move per call:

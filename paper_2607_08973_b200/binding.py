@@ -52,6 +52,8 @@ def lib() -> ctypes.CDLL:
             "sifar_slot_count": (sz, [ci, sz]),
             "sifar_algorithmic_bytes": (sz, [ci, ci, sz, ci]),
             "sifar_last_error": (ctypes.c_char_p, []),
+            "sifar_allreduce_noalloc": (ci, [vp, ci, vp, sz, ci, vp]),
+            "sifar_noalloc_max_elems": (sz, []),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -142,6 +144,15 @@ def sifar_slot_count(dtype: int, n: int) -> int:
 
 def sifar_algorithmic_bytes(P: int, dtype: int, n: int, mode: int) -> int:
     return lib().sifar_algorithmic_bytes(P, dtype, n, mode)
+
+
+def sifar_allreduce_noalloc(rank_ptrs, out: int, n: int, dtype: int, stream: int = 0) -> int:
+    """All-reduce of ready plain partials for callers that must not allocate (see include/sifar.h)."""
+    return _check(lib().sifar_allreduce_noalloc(_ptr_array(rank_ptrs), len(rank_ptrs), out, n, dtype, stream))
+
+
+def sifar_noalloc_max_elems() -> int:
+    return lib().sifar_noalloc_max_elems()
 
 
 # ---------------------------------------------------------------------------
