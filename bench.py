@@ -40,6 +40,8 @@ sys.path.insert(0, ROOT)
 METRIC = "p50 us per P=8 emulated all-reduce (decode payload), with HBM roofline fraction at a 16 MiB payload"
 P, HIDDEN, ARS_PER_STEP = 8, 4096, 64
 LARGE_N = 8 << 20                      # 16 MiB of bf16 per rank
+# DRAM bytes per launch of k_reduce_spec<bf16,8> at LARGE_N from one ncu capture: 179.01 MB read + 11.40 MB written
+NCU_TRAFFIC_BYTES = 190_412_544
 
 
 def read_peaks() -> tuple[float, str]:
@@ -293,38 +295,42 @@ def run_gpu(args) -> None:
     windows = []
 
     # -- 1. the timed region: exactly K decode steps, persistent chain, speculative ------------------
-    main = Chain(sf, torch, synth, n, sf.SPECULATIVE, sf.CHAIN_PERSISTENT)
-    for _ in range(args.warmup):
-        main.run()
-    main.stream.synchronize()
-    dist.barrier()
-    torch.cuda.synchronize()
-    w0 = time.time()
-    secs = main.timed_runs(args.steps)
-    torch.cuda.synchronize()
-    dist.barrier()
-    windows.append((w0, time.time()))
-    secs = dist.max_over_ranks(secs)
-    iv = main.intervals_us(min(args.steps, 200))
-    p50, p99 = dist.max_over_ranks(pct(iv, 50)), dist.max_over_ranks(pct(iv, 99))
-    launches = sf.sifar_chain_launches_per_run(main.chain) * args.steps
-    stats = sf.sifar_get_stats(main.ctx)
-    main.close()
+    secs, p50, p99, launches = 0.0, 0.0, 0.0, 0
+    stats = {"calls": 0, "calls_with_retry": 0, "slot_reloads": 0}
+    if args.only != "roofline":
+        main = Chain(sf, torch, synth, n, sf.SPECULATIVE, sf.CHAIN_PERSISTENT)
+        for _ in range(args.warmup):
+            main.run()
+        main.stream.synchronize()
+        dist.barrier()
+        torch.cuda.synchronize()
+        w0 = time.time()
+        secs = main.timed_runs(args.steps)
+        torch.cuda.synchronize()
+        dist.barrier()
+        windows.append((w0, time.time()))
+        secs = dist.max_over_ranks(secs)
+        iv = main.intervals_us(min(args.steps, 200))
+        p50, p99 = dist.max_over_ranks(pct(iv, 50)), dist.max_over_ranks(pct(iv, 99))
+        launches = sf.sifar_chain_launches_per_run(main.chain) * args.steps
+        stats = sf.sifar_get_stats(main.ctx)
+        main.close()
 
     detail, roof, roof_decode, e2e, cpu = {}, None, None, None, None
-    if rank == 0:
+    if rank == 0 and args.only != "decode":
         # -- 2. every mode and chain implementation on the same step, interleaved -------------------
         w0 = time.time()
         modes = (sf.BARRIER_ONESHOT, sf.DUALBUF, sf.SPECULATIVE, sf.CHAIN_NO_ALLREDUCE)
-        detail["modes"] = measure_modes(sf, torch, synth, n, args.warmup, max(8, args.steps // 8),
-                                        (sf.CHAIN_PERSISTENT, sf.CHAIN_GRAPH), modes)
-        if args.sweep:
+        impls = (sf.CHAIN_PERSISTENT,) if args.skip_graph else (sf.CHAIN_PERSISTENT, sf.CHAIN_GRAPH)
+        if args.only == "all":
+            detail["modes"] = measure_modes(sf, torch, synth, n, args.warmup, max(8, args.steps // 8), impls, modes)
+        if args.sweep and args.only == "all":
             detail["by_batch_tokens"] = {
                 str(b): measure_modes(sf, torch, synth, HIDDEN * b, args.warmup, max(8, args.steps // 8),
                                       (sf.CHAIN_PERSISTENT, sf.CHAIN_GRAPH), modes)
                 for b in (2, 4, 8, 16)}
             detail["streams"] = measure_modes(sf, torch, synth, n, 3, 8, (sf.CHAIN_STREAMS,), modes, rounds=2)
-        # -- 3. roofline: 16 MiB per rank, L2 flushed ------------------------------------------------
+        # -- 3. roofline: 16 MiB per rank, inputs larger than L2 -------------------------------------
         r_iters = max(5, min(20, args.steps))
         mean_s, med_s, cnt = measure_roofline(sf, torch, P, LARGE_N, sf.SPECULATIVE, 3, r_iters)
         alg = sf.sifar_algorithmic_bytes(P, sf.BF16, LARGE_N, sf.SPECULATIVE)
@@ -344,17 +350,15 @@ def run_gpu(args) -> None:
         ab = sf.sifar_algorithmic_bytes(P, sf.BF16, 4 * LARGE_N, sf.SPECULATIVE)
         roof["at_64MiB_per_rank"] = {"kernel_us": round(ms_ * 1e6, 2), "achieved": round(ab / ms_ / 1e9, 1),
                                      "frac": round(ab / ms_ / 1e9 / peak_gbs, 4)}
-        try:
-            with open(os.path.join(ROOT, "profiles", "traffic.json")) as fh:
-                roof["traffic"] = json.load(fh).get("k_reduce_spec_bf16_P8_n8Mi_dram_bytes")
-        except Exception:
-            pass
+        roof["traffic"] = NCU_TRAFFIC_BYTES
+        roof["traffic_source"] = "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel and size"
         alg_d = sf.sifar_algorithmic_bytes(P, sf.BF16, n, sf.SPECULATIVE) * ARS_PER_STEP
-        step_s = secs / args.steps
+        step_s = secs / args.steps if secs else float("inf")
         roof_decode = {"bound": "latency", "kernel": "k_chain<bf16,P=8,speculative>", "achieved": round(alg_d / step_s / 1e9, 1),
                        "peak": peak_gbs, "unit": "GB/s", "frac": round(alg_d / step_s / 1e9 / peak_gbs, 5),
                        "note": "decode payloads are L2-resident and latency-bound; see detail.modes"}
         windows.append((w0, time.time()))
+    if rank == 0 and args.only == "all":
         # -- 4. end to end through host buffers ------------------------------------------------------
         w0 = time.time()
         per_call = measure_e2e(sf, torch, synth, n, sf.SPECULATIVE, 2, max(4, min(args.steps, 20)))
@@ -413,6 +417,11 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="sifar", choices=["sifar", "reference"])
     ap.add_argument("--sweep", action="store_true", help="also batch sizes 2..16 and the stream chain")
+    ap.add_argument("--only", default="all", choices=["all", "decode", "roofline"],
+                    help="profiling aid: run the timed decode region only, or the roofline section only")
+    ap.add_argument("--skip-graph", action="store_true",
+                    help="profiling aid: leave out the graph / stream chains (under ncu kernels are serialised, and "
+                         "those chains' reducers wait for producers that run concurrently)")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = args.steps or 20
