@@ -1,0 +1,102 @@
+"""Parity at the full sizes of the workload list, in the launch configurations bench.py times."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_08973_b200 import binding as sf
+from paper_2607_08973_b200 import synth
+
+from gpu_util import BF16, F32, MODES, Ctx, allreduce_via_pack, assert_bits_equal, empty_out, out_to_numpy, to_device
+from test_gpu_chains import _oracle_w, _ring, _rows
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def skew_reference(oracle):
+    """Config 5 in full: 10 000 chained all-reduces of P=8, n=16384 integers, computed once by the oracle."""
+    d = synth.chain_workload("skew", 8)
+    return d, oracle.chain(_oracle_w(oracle, d), 8, 16384, BF16, 10_000)
+
+
+@pytest.mark.parametrize("impl,mode", [(sf.CHAIN_PERSISTENT, sf.SPECULATIVE), (sf.CHAIN_PERSISTENT, sf.DUALBUF),
+                                       (sf.CHAIN_PERSISTENT, sf.BARRIER_ONESHOT), (sf.CHAIN_GRAPH, sf.SPECULATIVE)])
+def test_config5_ten_thousand_skewed_steps(skew_reference, impl, mode):
+    d, want = skew_reference
+    P, n, steps, runs = 8, 16384, 100, 100
+    with Ctx(P, n, BF16, timeout_us=5_000_000) as ctx:
+        ring, stride = _ring(n, BF16, steps)
+        ch = sf.sifar_chain_create(ctx.h, sf.make_workload(**d), n, mode, impl, ring.data_ptr(), steps, steps)
+        try:
+            s = torch.cuda.Stream()
+            for k in range(runs):
+                sf.sifar_chain_run(ch, s.cuda_stream)
+                torch.cuda.synchronize()
+                assert sf.sifar_status(ctx.h) == 0
+                got = _rows(ring, stride, steps, n, BF16)
+                assert np.array_equal(got, want[k * steps:(k + 1) * steps]), f"segment {k}"
+            st = sf.sifar_get_stats(ctx.h)
+        finally:
+            sf.sifar_chain_destroy(ch)
+    assert st["calls"] == steps * runs and st["timeouts"] == 0
+    if mode == sf.SPECULATIVE:
+        assert 0 < st["calls_with_retry"] <= steps * runs and st["slot_reloads"] > 0
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_config4_largest_payload_every_mode(oracle, dtype):
+    """P=8, n=32 Mi (64 MiB of bf16 / 128 MiB of fp32 per rank): the whole output against the oracle."""
+    P, n = 8, 1 << 25
+    xs = synth.rank_inputs(P, n, dtype, 0x5EED0004, "uniform")
+    want = oracle.allreduce(xs, dtype)
+    xd = [to_device(x) for x in xs]
+    with Ctx(P, n, dtype) as ctx:
+        for mode in MODES:
+            out = empty_out(n, dtype)
+            torch.cuda.synchronize()
+            allreduce_via_pack(ctx, xd, n, mode, out)
+            torch.cuda.synchronize()
+            assert sf.sifar_status(ctx.h) == 0
+            got, tail = out_to_numpy(out, n, dtype)
+            assert_bits_equal(got, want, dtype, f"mode {mode}")
+            del out
+
+
+@pytest.mark.parametrize("P", [2, 4])
+def test_config4_sixteen_mib_other_rank_counts(oracle, P):
+    n = 1 << 23
+    xs = synth.rank_inputs(P, n, BF16, 0x5EED0004 + P, "uniform")
+    want = oracle.allreduce(xs, BF16)
+    xd = [to_device(x) for x in xs]
+    with Ctx(P, n, BF16) as ctx:
+        for mode in MODES:
+            out = empty_out(n, BF16)
+            torch.cuda.synchronize()
+            allreduce_via_pack(ctx, xd, n, mode, out)
+            torch.cuda.synchronize()
+            got, _ = out_to_numpy(out, n, BF16)
+            assert_bits_equal(got, want, BF16, f"P {P} mode {mode}")
+
+
+def test_large_payload_with_late_producers_uses_the_deferring_regime(oracle):
+    """Reducer enqueued first on a payload far larger than one CTA per SM; producers follow 300 us later."""
+    P, n = 8, 1 << 22
+    xs = synth.rank_inputs(P, n, BF16, 77, "uniform")
+    want = oracle.allreduce(xs, BF16)
+    xd = [to_device(x) for x in xs]
+    for mode in MODES:
+        with Ctx(P, n, BF16) as ctx:
+            out = empty_out(n, BF16)
+            ps = [torch.cuda.Stream() for _ in range(P)]
+            rs = torch.cuda.Stream()
+            torch.cuda.synchronize()
+            for r in range(P):
+                sf.sifar_spin(300_000, ps[r].cuda_stream)
+                sf.sifar_pack(ctx.h, r, xd[r].data_ptr(), n, mode, ps[r].cuda_stream)
+            sf.sifar_allreduce(ctx.h, None, out.data_ptr(), n, mode, rs.cuda_stream)
+            torch.cuda.synchronize()
+            assert sf.sifar_status(ctx.h) == 0
+            got, _ = out_to_numpy(out, n, BF16)
+            assert_bits_equal(got, want, BF16, f"mode {mode}")
+            st = sf.sifar_get_stats(ctx.h)
+            assert st["timeouts"] == 0 and st["calls"] == 1
