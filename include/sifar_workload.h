@@ -94,6 +94,22 @@ int sifar_chain_run(sifar_chain *chain, void *stream);
  */
 int sifar_chain_stamps(sifar_chain *chain, unsigned long long *stamps);
 
+/*
+ * Phase timeline of the persistent chain (the latency breakdown that stands in for
+ * a bandwidth figure at decode payloads).  enable != 0 makes later runs record,
+ * for every step s of a run, 32 %globaltimer stamps (0 = not taken) written by
+ * thread 0 of the CTAs that own chunk 0:
+ *   reducer:            [0] enters the step      [1] arrival flags seen (speculative: own slot valid)
+ *                       [2] whole chunk reduced  [3] ready flag released
+ *                       [28] done flags released (BARRIER_ONESHOT, last reducer CTA only)
+ *   producer of rank r: [4+3r] previous result's ready flag seen   [5+3r] stores issued
+ *                       [6+3r] arrival flag released (barrier modes)
+ * If `phases` is not NULL the stamps of the last run (steps_per_run x 32) are copied
+ * to it (synchronizes the device).  PERSISTENT chains with P = 2 or P = 8 only; the
+ * traced kernel is a separate build, so an untraced run pays nothing for it.
+ */
+int sifar_chain_trace(sifar_chain *chain, int enable, unsigned long long *phases);
+
 /* Kernels launched per run by this chain (graph replays count their kernel nodes). */
 int sifar_chain_launches_per_run(sifar_chain *chain);
 

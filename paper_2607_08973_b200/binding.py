@@ -189,6 +189,7 @@ def _wl() -> ctypes.CDLL:
             "sifar_chain_run": (ci, [vp, vp]),
             "sifar_chain_stamps": (ci, [vp, ullp]),
             "sifar_chain_launches_per_run": (ci, [vp]),
+            "sifar_chain_trace": (ci, [vp, ci, ullp]),
             "sifar_chain_destroy": (ci, [vp]),
             "sifar_workload_first": (ci, [wp, ci, ci, vp, sz, vp]),
             "sifar_workload_next": (ci, [wp, ci, cu, ci, vp, vp, sz, vp]),
@@ -223,6 +224,16 @@ def sifar_chain_stamps(chain: int, steps_per_run: int) -> list[int]:
     buf = (ctypes.c_ulonglong * (steps_per_run + 1))()
     _check(_wl().sifar_chain_stamps(chain, buf))
     return list(buf)
+
+
+def sifar_chain_trace(chain: int, enable: bool, steps_per_run: int = 0):
+    """Switches the phase trace on/off; with steps_per_run > 0 also returns the last run's [steps][40] stamps."""
+    if steps_per_run:
+        buf = (ctypes.c_ulonglong * (steps_per_run * 40))()
+        _check(_wl().sifar_chain_trace(chain, int(enable), buf))
+        return [list(buf[i * 40:(i + 1) * 40]) for i in range(steps_per_run)]
+    _check(_wl().sifar_chain_trace(chain, int(enable), None))
+    return None
 
 
 def sifar_chain_launches_per_run(chain: int) -> int:

@@ -115,10 +115,11 @@ template <int P> struct Unroll { static constexpr int value = (P <= 2) ? 4 : (P 
 template <int P, bool WIDE>
 __device__ __forceinline__ bool revalidate(uint4 (&x)[P], uint32_t stale, const uint4 *const *src, size_t s,
                                            uint32_t e, unsigned long long timeout_ns, uint32_t pace_ns,
-                                           unsigned &reloads)
+                                           unsigned &reloads, unsigned long long *round_stamps = nullptr)
 {
     Deadline d;
     bool burst = WIDE;
+    unsigned round = 0;
     do {
         /* issue every pending load before looking at any result, so that the re-loads overlap */
         const uint32_t pending = (WIDE || burst) ? stale : (stale & (0u - stale));
@@ -131,6 +132,8 @@ __device__ __forceinline__ bool revalidate(uint4 (&x)[P], uint32_t stale, const 
             if ((pending & (1u << r)) && x[r].w == e) stale &= ~(1u << r);
         reloads += __popc(pending);
         if (!WIDE) burst = !burst && stale != before;    /* the polled rank arrived: look at all others once */
+        if (round_stamps && round < 8u) round_stamps[round] = globaltimer_ns();
+        ++round;
         if (stale) {
             if (d.expired(timeout_ns)) return false;
             if (pace_ns) __nanosleep(pace_ns);
@@ -146,14 +149,15 @@ struct PollShape {
 
 template <int P>
 __device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const *src, size_t s, uint32_t e,
-                                              unsigned long long timeout_ns, PollShape shape, unsigned &reloads)
+                                              unsigned long long timeout_ns, PollShape shape, unsigned &reloads,
+                                              unsigned long long *round_stamps = nullptr)
 {
     uint32_t stale = 0;
 #pragma unroll
     for (int r = 0; r < P; ++r) stale |= (uint32_t)(x[r].w != e) << r;
     if (stale == 0u) return true;
-    return shape.wide ? revalidate<P, true>(x, stale, src, s, e, timeout_ns, shape.pace_ns, reloads)
-                      : revalidate<P, false>(x, stale, src, s, e, timeout_ns, shape.pace_ns, reloads);
+    return shape.wide ? revalidate<P, true>(x, stale, src, s, e, timeout_ns, shape.pace_ns, reloads, round_stamps)
+                      : revalidate<P, false>(x, stale, src, s, e, timeout_ns, shape.pace_ns, reloads, round_stamps);
 }
 
 /* ------------------------------------------------------------------------ */

@@ -362,10 +362,12 @@ struct PersistArgs {
     ChainDev *cs;
     ChunkFlags *chunks;
     unsigned long long *stamps;     /* steps + 1                           */
+    unsigned long long *trace;      /* NULL, or steps x kTraceSlots phase stamps of chunk 0 (see sifar_workload.h) */
     uint32_t *retry_steps;          /* steps: 1 if any CTA re-loaded a slot in that step */
 };
 
 constexpr int kChainThreads = 128;
+constexpr int kTraceSlots = 40;         /* 0-3 reducer, 4 + 3r .. 6 + 3r rank r's producer, 28 done flags */
 
 /* Bounded wait that also gives up when another CTA has already recorded a failure. */
 template <bool GE>
@@ -381,7 +383,7 @@ __device__ __forceinline__ bool chain_wait(const uint32_t *flag, uint32_t want, 
     }
 }
 
-template <int DT, int P, int MODE>
+template <int DT, int P, int MODE, bool TRACE>
 __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
 {
     DevState *st = a.st;
@@ -404,6 +406,9 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
     bool alive = true;
     const bool stamper = (blockIdx.x == 0);     /* reducer of chunk 0 (or rank 0's producer of chunk 0 without all-reduce) */
     if (stamper && threadIdx.x == 0) a.stamps[0] = globaltimer_ns();
+    /* phase trace: thread 0 of the reducer of chunk 0 and of rank 0's producer of chunk 0 */
+    const bool tracer = TRACE && a.trace != nullptr && threadIdx.x == 0 && chunk == 0;
+#define SIFAR_TRACE(slot) do { if (TRACE && tracer) a.trace[(size_t)s * kTraceSlots + (slot)] = globaltimer_ns(); } while (0)
 
     for (uint32_t s = 0; s < a.steps && alive; ++s) {
         const uint32_t e = a.e0 + 1u + s;
@@ -413,6 +418,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
 
         if (is_reducer) {
             /* ---------------- the pulling side ---------------- */
+            SIFAR_TRACE(0);
             const uint4 *src[P];
 #pragma unroll
             for (int r = 0; r < P; ++r) {
@@ -433,6 +439,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                 }
                 __syncthreads();
                 if (!s_ok) { alive = false; break; }
+                SIFAR_TRACE(1);
             }
             bool retried = false;
             for (uint32_t k = 0; k < a.K; ++k) {
@@ -443,12 +450,17 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                 for (int r = 0; r < P; ++r) x[r] = ld_slot(src[r] + u);
                 if (MODE == SIFAR_SPECULATIVE) {
                     const unsigned before = reloads;
-                    if (!validate_slot<P>(x, src, u, e, a.timeout_ns, a.poll, reloads)) {
+                    if (!validate_slot<P>(x, src, u, e, a.timeout_ns, a.poll, reloads,
+                                          (TRACE && tracer && k == 0) ? a.trace + (size_t)s * kTraceSlots + 30 : nullptr)) {
                         fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
                         alive = false;
                         break;
                     }
                     retried |= (reloads != before);
+                    if (k == 0) {
+                        SIFAR_TRACE(1);
+                        if (TRACE && tracer) a.trace[(size_t)s * kTraceSlots + 29] = reloads - before;
+                    }
                     store_slot_result<DT>(ring_row, u, n, sum_vec<DT, P>(x, false));
                 } else {
                     store_vec_result<DT>(ring_row, u, n, sum_vec<DT, P>(x, true));
@@ -458,8 +470,10 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                barrier of step s cannot race with the marks of step s + 1 */
             if (MODE == SIFAR_SPECULATIVE && retried) s_retried[s & 1u] = 1;
             if (!__syncthreads_and(alive)) { alive = false; break; }
+            SIFAR_TRACE(2);
             if (threadIdx.x == 0) {
                 st_release_u32(&cf->ready, e);                 /* result chunk published */
+                SIFAR_TRACE(3);
                 if (MODE == SIFAR_SPECULATIVE && s_retried[s & 1u]) {
                     s_retried[s & 1u] = 0;
                     st_relaxed_u32(&a.retry_steps[s], 1u);
@@ -470,6 +484,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                     const uint32_t arrived = atom_add_acq_rel_u32(&a.cs->bottom_count, 1u) + 1u;
                     if (arrived == a.bottom_base + (s + 1u) * C)
                         for (int r = 0; r < P; ++r) st_release_u32(&a.cs->done[r], e);
+                    SIFAR_TRACE(28);
                 }
             }
         } else {
@@ -494,6 +509,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                     if (ok && MODE == SIFAR_BARRIER_ONESHOT)
                         ok = chain_wait<true>(&a.cs->done[rank], e - 1u, st, a.host_status, a.timeout_ns);
                 }
+                SIFAR_TRACE(4 + 3 * rank);
                 if (ok) spin_ns(gen_delay_ns(a.w, rank, t));
                 s_ok = ok;
             }
@@ -519,9 +535,11 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                             make_uint4(w[0], w[1], w[2], w[NW - 1]));
                 }
             }
+            SIFAR_TRACE(5 + 3 * rank);
             if (MODE == SIFAR_BARRIER_ONESHOT || MODE == SIFAR_DUALBUF) {
                 __syncthreads();
                 if (threadIdx.x == 0) st_release_u32(&cf->arrive[p][rank], e);
+                SIFAR_TRACE(6 + 3 * rank);
             } else if (no_ar) {
                 __syncthreads();
                 if (stamper && threadIdx.x == 0) a.stamps[s + 1u] = globaltimer_ns();
@@ -529,6 +547,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
         }
     }
 
+#undef SIFAR_TRACE
     /* leave: mis-speculation counters, then the last CTA out publishes the call number */
     const unsigned warp_reloads = __reduce_add_sync(0xFFFFFFFFu, reloads);
     if (warp_reloads && (threadIdx.x & 31) == 0)
@@ -624,6 +643,8 @@ struct sifar_chain {
     ChainDev *d_cs;
     ChunkFlags *d_chunks;
     unsigned long long *d_stamps;
+    unsigned long long *d_trace;
+    int trace_on;
     uint32_t *d_retry_steps;
     uint32_t C, K;
     int grid;
@@ -722,36 +743,39 @@ static int enqueue_run(sifar_chain *ch, cudaStream_t origin, uint32_t first_t)
     return SIFAR_OK;
 }
 
-template <int DT, int P>
+template <int DT, int P, bool TRACE>
 static const void *chain_kernel_p(int mode)
 {
     switch (mode) {
-    case SIFAR_BARRIER_ONESHOT: return (const void *)k_chain<DT, P, SIFAR_BARRIER_ONESHOT>;
-    case SIFAR_DUALBUF:         return (const void *)k_chain<DT, P, SIFAR_DUALBUF>;
-    case SIFAR_SPECULATIVE:     return (const void *)k_chain<DT, P, SIFAR_SPECULATIVE>;
-    default:                    return (const void *)k_chain<DT, P, kModeNoAllreduce>;
+    case SIFAR_BARRIER_ONESHOT: return (const void *)k_chain<DT, P, SIFAR_BARRIER_ONESHOT, TRACE>;
+    case SIFAR_DUALBUF:         return (const void *)k_chain<DT, P, SIFAR_DUALBUF, TRACE>;
+    case SIFAR_SPECULATIVE:     return (const void *)k_chain<DT, P, SIFAR_SPECULATIVE, TRACE>;
+    default:                    return (const void *)k_chain<DT, P, kModeNoAllreduce, false>;
     }
 }
 
 template <int DT>
-static const void *chain_kernel_dt(int P, int mode)
+static const void *chain_kernel_dt(int P, int mode, bool trace)
 {
+    /* the traced build exists for the shapes of the workload list only */
+    if (trace && P == 8) return chain_kernel_p<DT, 8, true>(mode);
+    if (trace && P == 2) return chain_kernel_p<DT, 2, true>(mode);
     switch (P) {
-    case 1: return chain_kernel_p<DT, 1>(mode);
-    case 2: return chain_kernel_p<DT, 2>(mode);
-    case 3: return chain_kernel_p<DT, 3>(mode);
-    case 4: return chain_kernel_p<DT, 4>(mode);
-    case 5: return chain_kernel_p<DT, 5>(mode);
-    case 6: return chain_kernel_p<DT, 6>(mode);
-    case 7: return chain_kernel_p<DT, 7>(mode);
-    default: return chain_kernel_p<DT, 8>(mode);
+    case 1: return chain_kernel_p<DT, 1, false>(mode);
+    case 2: return chain_kernel_p<DT, 2, false>(mode);
+    case 3: return chain_kernel_p<DT, 3, false>(mode);
+    case 4: return chain_kernel_p<DT, 4, false>(mode);
+    case 5: return chain_kernel_p<DT, 5, false>(mode);
+    case 6: return chain_kernel_p<DT, 6, false>(mode);
+    case 7: return chain_kernel_p<DT, 7, false>(mode);
+    default: return chain_kernel_p<DT, 8, false>(mode);
     }
 }
 
-static const void *chain_kernel(const sifar_chain *ch)
+static const void *chain_kernel(const sifar_chain *ch, bool trace = false)
 {
-    return ch->ctx->dtype == SIFAR_BF16 ? chain_kernel_dt<SIFAR_BF16>(ch->ctx->P, ch->mode)
-                                        : chain_kernel_dt<SIFAR_F32>(ch->ctx->P, ch->mode);
+    return ch->ctx->dtype == SIFAR_BF16 ? chain_kernel_dt<SIFAR_BF16>(ch->ctx->P, ch->mode, trace)
+                                        : chain_kernel_dt<SIFAR_F32>(ch->ctx->P, ch->mode, trace);
 }
 
 static void chain_free(sifar_chain *ch)
@@ -768,6 +792,7 @@ static void chain_free(sifar_chain *ch)
     if (ch->d_cs) cudaFree(ch->d_cs);
     if (ch->d_chunks) cudaFree(ch->d_chunks);
     if (ch->d_stamps) cudaFree(ch->d_stamps);
+    if (ch->d_trace) cudaFree(ch->d_trace);
     if (ch->d_retry_steps) cudaFree(ch->d_retry_steps);
     delete ch;
 }
@@ -784,7 +809,8 @@ static int chain_setup_persistent(sifar_chain *ch)
     /* leave half of the machine free: the chain stands for a few operators of a forward pass, not all of it */
     const size_t budget = resident / 2 > (size_t)roles ? resident / 2 : (size_t)roles;
     uint32_t K = 1;
-    size_t C = (units + kChainThreads - 1) / kChainThreads;
+    if (const char *env = getenv("SIFAR_CHAIN_K")) K = (uint32_t)atoi(env) > 0 ? (uint32_t)atoi(env) : 1;
+    size_t C = (units + (size_t)kChainThreads * K - 1) / ((size_t)kChainThreads * K);
     while (C * roles > budget) {
         ++K;
         C = (units + (size_t)kChainThreads * K - 1) / ((size_t)kChainThreads * K);
@@ -793,6 +819,8 @@ static int chain_setup_persistent(sifar_chain *ch)
     SIFAR_CUDA(cudaMalloc(&ch->d_cs, sizeof(ChainDev)));
     SIFAR_CUDA(cudaMalloc(&ch->d_chunks, sizeof(ChunkFlags) * C));
     SIFAR_CUDA(cudaMalloc(&ch->d_stamps, sizeof(unsigned long long) * (ch->steps + 1)));
+    SIFAR_CUDA(cudaMalloc(&ch->d_trace, sizeof(unsigned long long) * ch->steps * kTraceSlots));
+    SIFAR_CUDA(cudaMemset(ch->d_trace, 0, sizeof(unsigned long long) * ch->steps * kTraceSlots));
     SIFAR_CUDA(cudaMalloc(&ch->d_retry_steps, sizeof(uint32_t) * ch->steps));
     SIFAR_CUDA(cudaMemset(ch->d_cs, 0, sizeof(ChainDev)));
     SIFAR_CUDA(cudaMemset(ch->d_chunks, 0, sizeof(ChunkFlags) * C));
@@ -902,8 +930,9 @@ extern "C" int sifar_chain_run(sifar_chain *ch, void *stream)
         a.bottom_base = ch->runs * (uint32_t)ch->steps * ch->C;
         a.exit_base = ch->runs * (uint32_t)ch->grid;
         a.cs = ch->d_cs; a.chunks = ch->d_chunks; a.stamps = ch->d_stamps; a.retry_steps = ch->d_retry_steps;
+        a.trace = ch->trace_on ? ch->d_trace : nullptr;
         void *params[] = {&a};
-        SIFAR_CUDA(cudaLaunchCooperativeKernel(chain_kernel(ch), dim3((unsigned)ch->grid), dim3(kChainThreads),
+        SIFAR_CUDA(cudaLaunchCooperativeKernel(chain_kernel(ch, ch->trace_on != 0), dim3((unsigned)ch->grid), dim3(kChainThreads),
                                                params, 0, s));
     }
     ch->runs += 1;
@@ -920,6 +949,25 @@ extern "C" int sifar_chain_stamps(sifar_chain *ch, unsigned long long *stamps)
     }
     SIFAR_CUDA(cudaDeviceSynchronize());
     SIFAR_CUDA(cudaMemcpy(stamps, ch->d_stamps, sizeof(unsigned long long) * (ch->steps + 1), cudaMemcpyDeviceToHost));
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_chain_trace(sifar_chain *ch, int enable, unsigned long long *phases)
+{
+    if (!ch || ch->impl != SIFAR_CHAIN_PERSISTENT) {
+        set_error("sifar_chain_trace: needs a persistent chain");
+        return SIFAR_ERR_INVALID;
+    }
+    if (enable && ch->ctx->P != 8 && ch->ctx->P != 2) {
+        set_error("sifar_chain_trace: the traced kernel is built for P = 2 and P = 8 only");
+        return SIFAR_ERR_INVALID;
+    }
+    ch->trace_on = enable ? 1 : 0;
+    if (phases) {
+        SIFAR_CUDA(cudaDeviceSynchronize());
+        SIFAR_CUDA(cudaMemcpy(phases, ch->d_trace, sizeof(unsigned long long) * ch->steps * kTraceSlots,
+                              cudaMemcpyDeviceToHost));
+    }
     return SIFAR_OK;
 }
 

@@ -192,3 +192,28 @@ def test_sixteen_byte_accesses_are_not_torn():
     torn, reads = sf.sifar_tear_check(1 << 16, 2000)
     assert reads >= (1 << 16) * 1000
     assert torn == 0
+
+
+def test_phase_trace_orders_the_phases_of_a_step():
+    """The traced build records the per-step timeline; phases of one step appear in protocol order."""
+    P, n, steps = 8, 4096, 64
+    _, d = _workloads("llama", P)
+    with Ctx(P, n, BF16) as ctx:
+        ring, _ = _ring(n, BF16, 2)
+        for mode in MODES:
+            ch = sf.sifar_chain_create(ctx.h, sf.make_workload(**d), n, mode, sf.CHAIN_PERSISTENT, ring.data_ptr(), 2, steps)
+            sf.sifar_chain_trace(ch, True)
+            sf.sifar_chain_run(ch, 0)
+            T = np.array(sf.sifar_chain_trace(ch, True, steps), dtype=np.int64)[2:]
+            assert sf.sifar_status(ctx.h) == 0
+            entered, seen, reduced, released = T[:, 0], T[:, 1], T[:, 2], T[:, 3]
+            assert np.all(entered <= seen) and np.all(seen <= reduced) and np.all(reduced <= released)
+            for r in range(P):
+                ready, stored = T[:, 4 + 3 * r], T[:, 5 + 3 * r]
+                assert np.all(ready <= stored)
+                assert np.all(stored <= reduced)                  # no result before every rank has stored
+                assert np.all(released[:-1] <= ready[1:])         # producers wait for the previous result
+                if mode != sf.SPECULATIVE:
+                    assert np.all(stored <= T[:, 6 + 3 * r]) and np.all(T[:, 6 + 3 * r] <= seen)
+            sf.sifar_chain_destroy(ch)
+            sf.sifar_reset(ctx.h, 0)
