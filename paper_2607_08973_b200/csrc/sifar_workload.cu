@@ -358,6 +358,7 @@ struct PersistArgs {
     uint32_t C;                     /* chunks = reducer CTAs               */
     uint32_t K;                     /* units per thread and step           */
     uint32_t bottom_base, exit_base;
+    uint32_t clustered;             /* role layout, see k_chain */
     PollShape poll;
     ChainDev *cs;
     ChunkFlags *chunks;
@@ -389,10 +390,26 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
     DevState *st = a.st;
     const uint32_t C = a.C;
     const bool no_ar = (MODE == kModeNoAllreduce);
-    const bool is_reducer = !no_ar && blockIdx.x < C;
-    const uint32_t pidx = no_ar ? blockIdx.x : blockIdx.x - C;
-    const uint32_t rank = is_reducer ? 0u : pidx / C;
-    const uint32_t chunk = is_reducer ? blockIdx.x : pidx % C;
+    /*
+     * Roles.  Clustered layout: the CTAs that own one chunk (its reducer and its P producers) are consecutive
+     * and launched as one thread-block cluster, which the hardware places inside one GPC, so their flag
+     * and slot traffic stays on one die.  Nothing else of the cluster is used: all communication still
+     * goes through global memory.  Flat layout: reducers first, then the producers rank by rank.
+     */
+    const uint32_t roles = no_ar ? (uint32_t)P : (uint32_t)P + 1u;
+    bool is_reducer;
+    uint32_t rank, chunk;
+    if (a.clustered) {
+        const uint32_t role = blockIdx.x % roles;
+        chunk = blockIdx.x / roles;
+        is_reducer = !no_ar && role == 0u;
+        rank = no_ar ? role : (is_reducer ? 0u : role - 1u);
+    } else {
+        is_reducer = !no_ar && blockIdx.x < C;
+        const uint32_t pidx = no_ar ? blockIdx.x : blockIdx.x - C;
+        rank = is_reducer ? 0u : pidx / C;
+        chunk = is_reducer ? blockIdx.x : pidx % C;
+    }
     ChunkFlags *cf = a.chunks + chunk;
     const size_t n = (size_t)a.n;
     constexpr int EPU = (MODE == SIFAR_SPECULATIVE) ? ((DT == SIFAR_BF16) ? 6 : 3) : ((DT == SIFAR_BF16) ? 8 : 4);
@@ -648,6 +665,7 @@ struct sifar_chain {
     uint32_t *d_retry_steps;
     uint32_t C, K;
     int grid;
+    bool clustered;                 /* one thread-block cluster per chunk (placement only) */
 };
 
 static bool valid_workload(const sifar_workload *w)
@@ -816,6 +834,29 @@ static int chain_setup_persistent(sifar_chain *ch)
         C = (units + (size_t)kChainThreads * K - 1) / ((size_t)kChainThreads * K);
     }
     ch->K = K; ch->C = (uint32_t)C; ch->grid = (int)(C * roles);
+    /* One cluster per chunk if the device can hold all of them at once (set SIFAR_CHAIN_CLUSTER=0 for the flat layout). */
+    ch->clustered = false;
+    const char *env_cluster = getenv("SIFAR_CHAIN_CLUSTER");
+    if (!(env_cluster && atoi(env_cluster) == 0) && roles <= 16) {
+        const void *fn = chain_kernel(ch);
+        cudaError_t err = cudaSuccess;
+        if (roles > 8) err = cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3((unsigned)ch->grid);
+        cfg.blockDim = dim3(kChainThreads);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)roles;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int max_clusters = 0;
+        if (err == cudaSuccess) err = cudaOccupancyMaxActiveClusters(&max_clusters, fn, &cfg);
+        if (err == cudaSuccess && (size_t)max_clusters >= C) ch->clustered = true;
+        else cudaGetLastError();
+    }
     SIFAR_CUDA(cudaMalloc(&ch->d_cs, sizeof(ChainDev)));
     SIFAR_CUDA(cudaMalloc(&ch->d_chunks, sizeof(ChunkFlags) * C));
     SIFAR_CUDA(cudaMalloc(&ch->d_stamps, sizeof(unsigned long long) * (ch->steps + 1)));
@@ -931,9 +972,30 @@ extern "C" int sifar_chain_run(sifar_chain *ch, void *stream)
         a.exit_base = ch->runs * (uint32_t)ch->grid;
         a.cs = ch->d_cs; a.chunks = ch->d_chunks; a.stamps = ch->d_stamps; a.retry_steps = ch->d_retry_steps;
         a.trace = ch->trace_on ? ch->d_trace : nullptr;
+        a.clustered = ch->clustered ? 1u : 0u;
         void *params[] = {&a};
-        SIFAR_CUDA(cudaLaunchCooperativeKernel(chain_kernel(ch, ch->trace_on != 0), dim3((unsigned)ch->grid), dim3(kChainThreads),
-                                               params, 0, s));
+        const void *fn = chain_kernel(ch, ch->trace_on != 0);
+        if (ch->clustered) {
+            const unsigned roles = (unsigned)(no_ar ? c->P : c->P + 1);
+            if (roles > 8) SIFAR_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+            cudaLaunchConfig_t cfg;
+            memset(&cfg, 0, sizeof cfg);
+            cfg.gridDim = dim3((unsigned)ch->grid);
+            cfg.blockDim = dim3(kChainThreads);
+            cfg.stream = s;
+            cudaLaunchAttribute attr[2];
+            attr[0].id = cudaLaunchAttributeCooperative;
+            attr[0].val.cooperative = 1;
+            attr[1].id = cudaLaunchAttributeClusterDimension;
+            attr[1].val.clusterDim.x = roles;
+            attr[1].val.clusterDim.y = 1;
+            attr[1].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 2;
+            SIFAR_CUDA(cudaLaunchKernelExC(&cfg, fn, params));
+        } else {
+            SIFAR_CUDA(cudaLaunchCooperativeKernel(fn, dim3((unsigned)ch->grid), dim3(kChainThreads), params, 0, s));
+        }
     }
     ch->runs += 1;
     if (!no_ar) c->h_epoch += (uint32_t)ch->steps;
