@@ -365,7 +365,9 @@ def run_gpu(args) -> None:
         windows.append((w0, time.time()))
         e2e = {"value": round(pct(per_call, 50), 2), "unit": "us", "p99": round(pct(per_call, 99), 2),
                "h2d_bytes_per_step": ARS_PER_STEP * P * n * 2, "d2h_bytes_per_step": ARS_PER_STEP * n * 2,
-               "what": "sifar_allreduce_host: pinned host partials -> H2D -> pack -> reduce -> D2H, per call"}
+               "what": "sifar_allreduce_host on pinned host buffers: one kernel packs the 8 partials straight from "
+                       "host memory (H2D inside the kernel), one reduces and writes the result to host memory, then "
+                       "a stream synchronisation; per call"}
         # -- 5. CPU oracle ---------------------------------------------------------------------------
         from oracle import oracle
         ar_us, reps = oracle_allreduce_us(oracle, synth, n, 6.0)

@@ -20,6 +20,13 @@
  * for r = 1..P-1 in binary32, round-to-nearest-even;  out[i] = narrow(acc) with
  * one RNE to the element type.
  *
+ * Tuning knobs, read from the environment by sifar_create / sifar_chain_create
+ * (defaults are what measurement on B200 settled on):
+ *   SIFAR_SPIN_NS           how long a CTA of a large reducer grid waits before it queues its tile (5000)
+ *   SIFAR_POLL_WIDE_MAX     re-poll all stale ranks per round up to this many (slot, rank) pairs (16384)
+ *   SIFAR_POLL_PACE_NS/_MIN sleep between polling rounds above _MIN pairs (0 = unpaced)
+ *   SIFAR_CHAIN_CLUSTER     0 = persistent chain without thread-block clusters
+ *
  * All pointers named "device" are CUDA device pointers valid on the context's
  * device; "stream" arguments are cudaStream_t passed as void* (NULL = the legacy
  * default stream).  Functions return a sifar_status_t unless stated otherwise;
@@ -106,10 +113,13 @@ int sifar_allreduce(sifar_ctx *ctx, const void *const *rank_ptrs, void *out, siz
                     int mode, void *stream);
 
 /*
- * Same operation from HOST memory, synchronous: copies the P host partials
- * (n plain elements each) to the device, packs them, reduces, copies the result
- * to host_out and waits.  Uses staging buffers the context allocates on the first
- * such call.  For end-to-end measurements and simple clients.
+ * Same operation from HOST memory, synchronous: moves the P host partials
+ * (n plain elements each) to the device, packs them, reduces, delivers the result
+ * in host_out and waits.  Pinned (page-locked), 16-byte aligned buffers are read
+ * and written in place by the kernels: one launch packs all ranks, one reduces.
+ * Pageable buffers go through staging buffers that the context allocates on the
+ * first such call (one copy per rank).  For end-to-end measurements and simple
+ * clients.
  */
 int sifar_allreduce_host(sifar_ctx *ctx, const void *const *host_rank_ptrs, void *host_out,
                          size_t n, int mode);

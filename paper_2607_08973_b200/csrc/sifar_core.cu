@@ -446,7 +446,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
 /* producer-side store path                                                  */
 /* ------------------------------------------------------------------------ */
 template <int DT, int MODE>
-__global__ void __launch_bounds__(kThreads) k_pack(const PackArgs a)
+__device__ __forceinline__ void pack_body(const PackArgs &a)
 {
     DevState *st = a.st;
     __shared__ uint32_t s_epoch;
@@ -507,6 +507,29 @@ __global__ void __launch_bounds__(kThreads) k_pack(const PackArgs a)
             store_slot(slots, s, w[0], w[1], w[2], e);
         }
     }
+}
+
+template <int DT, int MODE>
+__global__ void __launch_bounds__(kThreads) k_pack(const PackArgs a)
+{
+    pack_body<DT, MODE>(a);
+}
+
+/* All P ranks in one launch (blockIdx.y = rank): the host-buffer entry point packs straight from pinned host memory. */
+struct PackAllArgs {
+    const void *src[kMaxRanks];
+    void *dst[kMaxRanks];
+    PackArgs common;             /* src, dst and rank are filled in per rank */
+};
+
+template <int DT, int MODE>
+__global__ void __launch_bounds__(kThreads) k_pack_all(const PackAllArgs all)
+{
+    PackArgs a = all.common;
+    a.rank = blockIdx.y;
+    a.src = all.src[blockIdx.y];
+    a.dst = all.dst[blockIdx.y];
+    pack_body<DT, MODE>(a);
 }
 
 /* Release of one rank's arrival flag after caller-written plain partials. */
@@ -631,6 +654,17 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
         : launch_reduce_dt<SIFAR_F32>(ctx->P, rl.mode, (int)ntiles, stream, a);
     SIFAR_CUDA(err);
     return SIFAR_OK;
+}
+
+template <int DT>
+static cudaError_t launch_pack_all_dt(int mode, dim3 grid, cudaStream_t s, const PackAllArgs &a)
+{
+    switch (mode) {
+    case SIFAR_BARRIER_ONESHOT: k_pack_all<DT, SIFAR_BARRIER_ONESHOT><<<grid, kThreads, 0, s>>>(a); break;
+    case SIFAR_DUALBUF:         k_pack_all<DT, SIFAR_DUALBUF><<<grid, kThreads, 0, s>>>(a); break;
+    default:                    k_pack_all<DT, SIFAR_SPECULATIVE><<<grid, kThreads, 0, s>>>(a); break;
+    }
+    return cudaGetLastError();
 }
 
 template <int DT>
@@ -959,6 +993,16 @@ extern "C" int sifar_debug_set_epoch(sifar_ctx *c, unsigned calls_so_far)
     return SIFAR_OK;
 }
 
+/* Device-usable address of a host pointer if it is pinned (or otherwise reachable from the GPU), else NULL. */
+static void *device_view(const void *p)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeManaged || at.type == cudaMemoryTypeDevice)
+        return at.devicePointer;
+    return nullptr;
+}
+
 extern "C" int sifar_allreduce_host(sifar_ctx *c, const void *const *host_rank_ptrs, void *host_out, size_t n,
                                     int mode)
 {
@@ -968,10 +1012,61 @@ extern "C" int sifar_allreduce_host(sifar_ctx *c, const void *const *host_rank_p
         set_error("sifar_allreduce_host: bad mode, n or pointer");
         return SIFAR_ERR_INVALID;
     }
+    for (int r = 0; r < c->P; ++r)
+        if (!host_rank_ptrs[r]) { set_error("sifar_allreduce_host: NULL rank pointer"); return SIFAR_ERR_INVALID; }
+    cudaStream_t s = c->host_stream;
+    const size_t bytes = n * elem_size(c->dtype);
+
+    /* Fast path: every partial is pinned host memory the GPU can read in place.  One kernel packs all P
+       ranks straight from host memory (the H2D transfer happens inside that kernel), one reduces. */
+    PackAllArgs all;
+    memset(&all, 0, sizeof all);
+    bool direct = (n > 0);
+    for (int r = 0; r < c->P && direct; ++r) {
+        void *d = device_view(host_rank_ptrs[r]);
+        direct = d && (((uintptr_t)d & 15u) == 0);
+        all.src[r] = d;
+    }
+    if (direct) {
+        uint32_t e;
+        if ((rc = next_epoch(c, "sifar_allreduce_host", &e))) return rc;
+        for (int r = 0; r < c->P; ++r) all.dst[r] = const_cast<void *>(ctx_buffer(c, mode, e, r));
+        all.common.n = n;
+        all.common.st = c->d_state;
+        all.common.host_status = c->d_status_alias;
+        all.common.timeout_ns = c->timeout_ns;
+        all.common.parity = e & 1u;
+        all.common.wait_delta = (mode == SIFAR_BARRIER_ONESHOT && c->last_mode0_epoch) ? e - c->last_mode0_epoch : 0u;
+        const size_t units = (mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, n) : (bytes + 15) / 16;
+        size_t gx = (units + kThreads - 1) / kThreads;
+        const size_t cap = (size_t)c->sm_count * 2;
+        if (gx > cap) gx = cap;
+        cudaError_t err = (c->dtype == SIFAR_BF16)
+            ? launch_pack_all_dt<SIFAR_BF16>(mode, dim3((unsigned)gx, (unsigned)c->P), s, all)
+            : launch_pack_all_dt<SIFAR_F32>(mode, dim3((unsigned)gx, (unsigned)c->P), s, all);
+        SIFAR_CUDA(err);
+        void *out_dev = device_view(host_out);
+        if (out_dev && ((uintptr_t)out_dev & 15u) == 0) {
+            if ((rc = sifar_allreduce(c, nullptr, out_dev, n, mode, s))) return rc;     /* result written in place */
+        } else {
+            if (!c->d_stage_out) {
+                cudaError_t e2 = cudaMalloc(&c->d_stage_out, c->plain_stride);
+                if (e2 != cudaSuccess) { cudaGetLastError(); set_error("sifar_allreduce_host: staging allocation failed"); return SIFAR_ERR_NOMEM; }
+            }
+            if ((rc = sifar_allreduce(c, nullptr, c->d_stage_out, n, mode, s))) return rc;
+            SIFAR_CUDA(cudaMemcpyAsync(host_out, c->d_stage_out, bytes, cudaMemcpyDeviceToHost, s));
+        }
+        SIFAR_CUDA(cudaStreamSynchronize(s));
+        rc = *c->h_status;
+        if (rc) set_error("sifar_allreduce_host: device status %d", rc);
+        return rc;
+    }
+
+    /* General path: pageable host memory goes through staging buffers allocated on first use. */
     const size_t stride = c->plain_stride;
     if (!c->d_stage_in) {
         cudaError_t e = cudaMalloc(&c->d_stage_in, stride * c->P);
-        if (e == cudaSuccess) e = cudaMalloc(&c->d_stage_out, stride);
+        if (e == cudaSuccess && !c->d_stage_out) e = cudaMalloc(&c->d_stage_out, stride);
         if (e != cudaSuccess) {
             if (c->d_stage_in) { cudaFree(c->d_stage_in); c->d_stage_in = nullptr; }
             cudaGetLastError();
@@ -979,10 +1074,7 @@ extern "C" int sifar_allreduce_host(sifar_ctx *c, const void *const *host_rank_p
             return SIFAR_ERR_NOMEM;
         }
     }
-    cudaStream_t s = c->host_stream;
-    const size_t bytes = n * elem_size(c->dtype);
     for (int r = 0; r < c->P; ++r) {
-        if (!host_rank_ptrs[r]) { set_error("sifar_allreduce_host: NULL rank pointer"); return SIFAR_ERR_INVALID; }
         if (bytes) SIFAR_CUDA(cudaMemcpyAsync(c->d_stage_in + r * stride, host_rank_ptrs[r], bytes, cudaMemcpyHostToDevice, s));
         if ((rc = sifar_pack(c, r, c->d_stage_in + r * stride, n, mode, s))) return rc;
     }

@@ -115,7 +115,6 @@ struct ReduceLaunch {
     size_t n;
     int mode;
     uint32_t parity;                 /* parity the host expects the call number to have */
-    int use_flags;                   /* barrier modes: poll arrival flags               */
 };
 
 int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream);

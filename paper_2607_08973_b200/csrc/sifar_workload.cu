@@ -711,8 +711,7 @@ static int enqueue_run(sifar_chain *ch, cudaStream_t origin, uint32_t first_t)
     const size_t units = (ch->mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, ch->n)
                                                          : (ch->n * elem_size(c->dtype) + 15) / 16;
     size_t pgrid = (units + kProdThreads - 1) / kProdThreads;
-    size_t cap = (size_t)c->sm_count * 2;
-    if (const char *env = getenv("SIFAR_PROD_CAP")) cap = (size_t)atoi(env);
+    const size_t cap = (size_t)c->sm_count * 2;
     if (pgrid > cap) pgrid = cap;
 
     for (int s = 0; s < ch->steps; ++s) {
@@ -826,9 +825,8 @@ static int chain_setup_persistent(sifar_chain *ch)
     const size_t resident = (size_t)per_sm * c->sm_count;
     /* leave half of the machine free: the chain stands for a few operators of a forward pass, not all of it */
     const size_t budget = resident / 2 > (size_t)roles ? resident / 2 : (size_t)roles;
-    uint32_t K = 1;
-    if (const char *env = getenv("SIFAR_CHAIN_K")) K = (uint32_t)atoi(env) > 0 ? (uint32_t)atoi(env) : 1;
-    size_t C = (units + (size_t)kChainThreads * K - 1) / ((size_t)kChainThreads * K);
+    uint32_t K = 1;      /* units per thread and step: 1 whenever the grid fits (more only lengthens the step) */
+    size_t C = (units + kChainThreads - 1) / kChainThreads;
     while (C * roles > budget) {
         ++K;
         C = (units + (size_t)kChainThreads * K - 1) / ((size_t)kChainThreads * K);

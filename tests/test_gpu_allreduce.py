@@ -145,14 +145,23 @@ def test_shrinking_then_growing_payload(oracle):
             assert_bits_equal(got, oracle.allreduce(xs, BF16), BF16, f"call {call} n {n}")
 
 
-def test_host_buffer_entry_point(oracle):
-    P, n = 8, 50_001
-    with Ctx(P, n, BF16) as ctx:
-        for mode in MODES:
-            xs = synth.rank_inputs(P, n, BF16, 77 + mode, "gauss")
-            out = np.zeros(n, dtype=np.uint16)
-            sf.sifar_allreduce_host(ctx.h, [x.ctypes.data for x in xs], out.ctypes.data, n, mode)
-            assert_bits_equal(out, oracle.allreduce(xs, BF16), BF16, f"host mode {mode}")
+@pytest.mark.parametrize("pinned", [False, True])
+def test_host_buffer_entry_point(oracle, pinned):
+    """Pageable buffers take the staging path, pinned ones are read and written in place by the kernels."""
+    P = 8
+    with Ctx(P, 50_001, BF16) as ctx:
+        for n in (50_001, 4096, 7):
+            for mode in MODES:
+                xs = synth.rank_inputs(P, n, BF16, 77 + mode + n, "gauss")
+                if pinned:
+                    hx = [torch.from_numpy(x.view(np.int16).copy()).pin_memory() for x in xs]
+                    hout = torch.zeros(n, dtype=torch.int16).pin_memory()
+                    sf.sifar_allreduce_host(ctx.h, [t.data_ptr() for t in hx], hout.data_ptr(), n, mode)
+                    out = hout.numpy().view(np.uint16)
+                else:
+                    out = np.zeros(n, dtype=np.uint16)
+                    sf.sifar_allreduce_host(ctx.h, [x.ctypes.data for x in xs], out.ctypes.data, n, mode)
+                assert_bits_equal(out, oracle.allreduce(xs, BF16), BF16, f"host pinned={pinned} n={n} mode {mode}")
 
 
 def test_argument_validation():
