@@ -313,6 +313,14 @@ __device__ __forceinline__ Roles cta_arrive(const ReduceArgs &a, uint32_t e, int
                 if ((d.polls % 64u) == 0u && ld_relaxed_u32(&st->status) != 0u) { r.ok = 0u; break; }
             }
             r.ndefer = ld_relaxed_u32(a.defer);
+            if (r.ok && r.ndefer == 0u) {
+                /* Nothing was queued (the usual case): janitor 1 publishes at once, the others just leave. */
+                if (r.janitor == 1u) {
+                    st_relaxed_u32(&st->cta_arrive, 0u);
+                    publish_call<MODE>(st, e, P);
+                }
+                r.janitor = 0u;
+            }
         }
         s_roles = r;
     }
