@@ -279,6 +279,30 @@ def measure_e2e(sf, torch, synth, n, mode, warmup, steps):
     return np.asarray(per_call) * 1e6
 
 
+def payload_sweep(sf, torch, exps=range(10, 26), ranks=(2, 4, 8)):
+    """Config 4: reducer time against payload, data ready, every mode; bf16 for all P, fp32 for P = 8.
+
+    Per point: enough contexts that the partials exceed twice the L2 (at least 4, at most 24); their reducers
+    run back to back between two CUDA events; the figure is the median over repetitions of time / launches.
+    Small payloads are bound by the launch rate of back-to-back kernels, not by the kernel.
+    """
+    rows = []
+    for P_ in ranks:
+        for dtype in ((0, 1) if P_ == 8 else (0,)):
+            for ex in exps:
+                n = 1 << ex
+                per_call = P_ * n * (2 if dtype == 0 else 4)
+                nctx = int(min(24, max(4, (2 * 126e6) // max(per_call, 1) + 1)))
+                row = {"P": P_, "dtype": "bf16" if dtype == 0 else "f32", "n": n,
+                       "payload_bytes_per_rank": n * (2 if dtype == 0 else 4)}
+                for mode in (sf.BARRIER_ONESHOT, sf.DUALBUF, sf.SPECULATIVE):
+                    mean_s, med_s, _ = measure_roofline(sf, torch, P_, n, mode, 2, 5, dtype=dtype, nctx=nctx)
+                    alg = sf.sifar_algorithmic_bytes(P_, dtype, n, mode)
+                    row[sf.MODE_NAMES[mode]] = {"us": round(med_s * 1e6, 2), "GBps": round(alg / med_s / 1e9, 1)}
+                rows.append(row)
+    return rows
+
+
 def run_gpu(args) -> None:
     import torch
     from paper_2607_08973_b200 import binding as sf
@@ -330,6 +354,7 @@ def run_gpu(args) -> None:
                                       (sf.CHAIN_PERSISTENT, sf.CHAIN_GRAPH), modes)
                 for b in (2, 4, 8, 16)}
             detail["streams"] = measure_modes(sf, torch, synth, n, 3, 8, (sf.CHAIN_STREAMS,), modes, rounds=2)
+            detail["payload_sweep"] = payload_sweep(sf, torch)
         # -- 3. roofline: 16 MiB per rank, inputs larger than L2 -------------------------------------
         r_iters = max(5, min(20, args.steps))
         mean_s, med_s, cnt = measure_roofline(sf, torch, P, LARGE_N, sf.SPECULATIVE, 3, r_iters)
