@@ -25,6 +25,7 @@
  *   SIFAR_SPIN_NS           how long a CTA of a large reducer grid waits before it queues its tile (5000)
  *   SIFAR_POLL_WIDE_MAX     re-poll all stale ranks per round up to this many (slot, rank) pairs (16384)
  *   SIFAR_POLL_PACE_NS/_MIN sleep between polling rounds above _MIN pairs (0 = unpaced)
+ *   SIFAR_POLL_SENTINEL_MIN persistent chain: above this many pairs a warp first waits on one slot per rank (16384)
  *   SIFAR_CHAIN_CLUSTER     0 = persistent chain without thread-block clusters
  *
  * All pointers named "device" are CUDA device pointers valid on the context's

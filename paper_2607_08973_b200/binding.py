@@ -227,11 +227,11 @@ def sifar_chain_stamps(chain: int, steps_per_run: int) -> list[int]:
 
 
 def sifar_chain_trace(chain: int, enable: bool, steps_per_run: int = 0):
-    """Switches the phase trace on/off; with steps_per_run > 0 also returns the last run's [steps][40] stamps."""
+    """Switches the phase trace on/off; with steps_per_run > 0 also returns the last run's [steps][48] stamps."""
     if steps_per_run:
-        buf = (ctypes.c_ulonglong * (steps_per_run * 40))()
+        buf = (ctypes.c_ulonglong * (steps_per_run * 48))()
         _check(_wl().sifar_chain_trace(chain, int(enable), buf))
-        return [list(buf[i * 40:(i + 1) * 40]) for i in range(steps_per_run)]
+        return [list(buf[i * 48:(i + 1) * 48]) for i in range(steps_per_run)]
     _check(_wl().sifar_chain_trace(chain, int(enable), None))
     return None
 

@@ -612,6 +612,7 @@ sifar::PollShape sifar::poll_shape_for(const sifar_ctx *ctx, size_t n)
     PollShape p;
     p.wide = pairs <= ctx->poll_wide_max ? 1u : 0u;
     p.pace_ns = pairs <= ctx->poll_pace_min ? 0u : ctx->poll_pace_ns;
+    p.sentinel = pairs <= ctx->poll_sentinel_min ? 0u : 1u;
     return p;
 }
 
@@ -735,6 +736,8 @@ extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
     c->spin_ns = 5000;
     if (const char *env = getenv("SIFAR_SPIN_NS")) c->spin_ns = strtoull(env, nullptr, 10);
     c->poll_pace_min = 16384;
+    c->poll_sentinel_min = 16384;
+    if (const char *env = getenv("SIFAR_POLL_SENTINEL_MIN")) c->poll_sentinel_min = (size_t)strtoull(env, nullptr, 10);
     c->poll_pace_ns = 0;
     if (const char *env = getenv("SIFAR_POLL_WIDE_MAX")) c->poll_wide_max = (size_t)strtoull(env, nullptr, 10);
     if (const char *env = getenv("SIFAR_POLL_PACE_MIN")) c->poll_pace_min = (size_t)strtoull(env, nullptr, 10);

@@ -87,6 +87,7 @@ struct sifar_ctx {
     size_t poll_wide_max;            /* speculative: wide polling up to this many (slot, rank) pairs per call */
     size_t poll_pace_min;            /* ... paced polling above this many pairs                              */
     uint32_t poll_pace_ns;
+    size_t poll_sentinel_min;        /* ... sentinel wait per warp above this many pairs (persistent chain) */
     /* staging for sifar_allreduce_host, allocated on first use */
     char *d_stage_in;
     char *d_stage_out;

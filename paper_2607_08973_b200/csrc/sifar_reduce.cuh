@@ -145,7 +145,37 @@ __device__ __forceinline__ bool revalidate(uint4 (&x)[P], uint32_t stale, const 
 struct PollShape {
     uint32_t wide;
     uint32_t pace_ns;
+    uint32_t sentinel;     /* wait on one slot per rank and warp before touching the warp's other slots */
 };
+
+/*
+ * Sentinel wait of a warp (all 32 lanes call): lane r < P polls rank r's copy of the warp's first slot
+ * until it carries the call number; the other lanes idle.  A producer warp writes 32 consecutive slots
+ * with one store instruction, so once the first is visible the rest follow within the same few hundred
+ * nanoseconds, and the warp's 32 x P bulk loads can go out and will almost always validate at once.
+ * Compared with every lane polling its own P slots this costs one extra L2 round trip after the last
+ * arrival, but it keeps 31/32 of the lines free of poll traffic while the producers are storing into
+ * them, which is what large waiting grids need.  Returns false on time-out (any lane).
+ */
+template <int P>
+__device__ __forceinline__ bool sentinel_wait(const uint4 *const *src, size_t warp_first_slot, uint32_t e,
+                                              unsigned long long timeout_ns, unsigned &reloads)
+{
+    const unsigned lane = threadIdx.x & 31u;
+    bool ok = true;
+    if (lane < (unsigned)P) {
+        const uint4 *p = nullptr;
+#pragma unroll
+        for (int r = 0; r < P; ++r)
+            if (lane == (unsigned)r) p = src[r] + warp_first_slot;
+        Deadline d;
+        while (ld_slot(p).w != e) {
+            ++reloads;
+            if (d.expired(timeout_ns)) { ok = false; break; }
+        }
+    }
+    return __all_sync(0xFFFFFFFFu, ok);
+}
 
 template <int P>
 __device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const *src, size_t s, uint32_t e,

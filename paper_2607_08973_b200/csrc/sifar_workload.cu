@@ -368,7 +368,7 @@ struct PersistArgs {
 };
 
 constexpr int kChainThreads = 128;
-constexpr int kTraceSlots = 40;         /* 0-3 reducer, 4 + 3r .. 6 + 3r rank r's producer, 28 done flags */
+constexpr int kTraceSlots = 48;         /* 0-3 reducer, 4 + 3r .. 6 + 3r rank r's producer, 28 done flags */
 
 /* Bounded wait that also gives up when another CTA has already recorded a failure. */
 template <bool GE>
@@ -461,6 +461,18 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
             bool retried = false;
             for (uint32_t k = 0; k < a.K; ++k) {
                 const size_t u = unit0 + (size_t)k * kChainThreads;
+                if (MODE == SIFAR_SPECULATIVE && a.poll.sentinel) {
+                    /* warp-uniform: the warp's first slot decides whether the warp has work at all */
+                    const size_t w0 = u - (threadIdx.x & 31u);
+                    if (w0 >= nunits) break;
+                    const unsigned before = reloads;
+                    if (!sentinel_wait<P>(src, w0, e, a.timeout_ns, reloads)) {
+                        if (threadIdx.x == 0 || (threadIdx.x & 31u) == 0u) fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+                        alive = false;
+                        break;
+                    }
+                    retried |= (reloads != before);
+                }
                 if (u >= nunits) break;
                 uint4 x[P];
 #pragma unroll
@@ -474,6 +486,8 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                         break;
                     }
                     retried |= (reloads != before);
+                    if (TRACE && a.trace != nullptr && chunk == 0 && k == 0 && (threadIdx.x & 31) == 0)
+                        a.trace[(size_t)s * kTraceSlots + 38 + (threadIdx.x >> 5)] = globaltimer_ns();
                     if (k == 0) {
                         SIFAR_TRACE(1);
                         if (TRACE && tracer) a.trace[(size_t)s * kTraceSlots + 29] = reloads - before;
@@ -552,6 +566,8 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                             make_uint4(w[0], w[1], w[2], w[NW - 1]));
                 }
             }
+            if (TRACE && a.trace != nullptr && chunk == 0 && rank == 0 && (threadIdx.x & 31) == 0)
+                a.trace[(size_t)s * kTraceSlots + 42 + (threadIdx.x >> 5)] = globaltimer_ns();
             SIFAR_TRACE(5 + 3 * rank);
             if (MODE == SIFAR_BARRIER_ONESHOT || MODE == SIFAR_DUALBUF) {
                 __syncthreads();
