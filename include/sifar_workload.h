@@ -64,7 +64,7 @@ typedef enum {
    A timing floor; its results are not a sum. */
 enum { SIFAR_CHAIN_NO_ALLREDUCE = 3 };
 
-/* Bytes between two rows of an output ring for n elements (a multiple of 256). */
+/* Bytes between two rows of an output ring for n elements (a multiple of 256, at least 16 bytes more than the row). */
 size_t sifar_chain_ring_stride(int dtype, size_t n);
 
 /*
@@ -88,11 +88,16 @@ int sifar_chain_run(sifar_chain *chain, void *stream);
 
 /*
  * Device timestamps (nanoseconds, %globaltimer) of the last run, after it has
- * finished: stamps[0] = start of the run, stamps[s] = result of step s of the run
- * published, s = 1..steps_per_run.  PERSISTENT only (else SIFAR_ERR_INVALID).
- * Synchronizes the device.
+ * finished: stamps[0] = start of the run (earliest CTA), stamps[s] = result of
+ * step s of the run complete, i.e. its last chunk published, s = 1..steps_per_run
+ * (the chunks of a result are reduced by different CTAs, which may run ahead of
+ * one another).  PERSISTENT only (else SIFAR_ERR_INVALID).  Synchronizes the device.
  */
 int sifar_chain_stamps(sifar_chain *chain, unsigned long long *stamps);
+
+/* The same stamps for one chunk alone (its reducer CTA), and the number of chunks of a PERSISTENT chain. */
+int sifar_chain_chunk_stamps(sifar_chain *chain, int chunk, unsigned long long *stamps);
+int sifar_chain_chunks(sifar_chain *chain);
 
 /*
  * Phase timeline of the persistent chain (the latency breakdown that stands in for

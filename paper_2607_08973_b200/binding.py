@@ -188,6 +188,8 @@ def _wl() -> ctypes.CDLL:
             "sifar_chain_create": (vp, [vp, wp, sz, ci, ci, vp, ci, ci]),
             "sifar_chain_run": (ci, [vp, vp]),
             "sifar_chain_stamps": (ci, [vp, ullp]),
+            "sifar_chain_chunk_stamps": (ci, [vp, ci, ullp]),
+            "sifar_chain_chunks": (ci, [vp]),
             "sifar_chain_launches_per_run": (ci, [vp]),
             "sifar_chain_trace": (ci, [vp, ci, ullp]),
             "sifar_chain_destroy": (ci, [vp]),
@@ -224,6 +226,16 @@ def sifar_chain_stamps(chain: int, steps_per_run: int) -> list[int]:
     buf = (ctypes.c_ulonglong * (steps_per_run + 1))()
     _check(_wl().sifar_chain_stamps(chain, buf))
     return list(buf)
+
+
+def sifar_chain_chunk_stamps(chain: int, chunk: int, steps_per_run: int) -> list[int]:
+    buf = (ctypes.c_ulonglong * (steps_per_run + 1))()
+    _check(_wl().sifar_chain_chunk_stamps(chain, chunk, buf))
+    return list(buf)
+
+
+def sifar_chain_chunks(chain: int) -> int:
+    return _wl().sifar_chain_chunks(chain)
 
 
 def sifar_chain_trace(chain: int, enable: bool, steps_per_run: int = 0):

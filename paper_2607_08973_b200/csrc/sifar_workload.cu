@@ -161,13 +161,15 @@ __device__ __forceinline__ float apply_update(const Gen &g, bool first, float pr
 
 template <int DT, int NW>
 __device__ __forceinline__ void unit_combine(const Gen &g, bool first, const void *prev, size_t i0, size_t n,
-                                             const float (&z)[NW * ((DT == SIFAR_BF16) ? 2 : 1)], uint32_t (&w)[NW])
+                                             const float (&z)[NW * ((DT == SIFAR_BF16) ? 2 : 1)], uint32_t (&w)[NW],
+                                             size_t n_readable = 0)
 {
     constexpr int EPW = (DT == SIFAR_BF16) ? 2 : 1;
     uint32_t pw[NW];
 #pragma unroll
     for (int j = 0; j < NW; ++j) pw[j] = 0u;
-    const bool full = (i0 + (size_t)NW * EPW <= n);
+    /* n_readable > n: the row behind `prev` is padded, so a ragged last unit can be loaded whole */
+    const bool full = (i0 + (size_t)NW * EPW <= (n_readable > n ? n_readable : n));
     if (!first) {
         if (full) {
             const uint32_t *p32 = reinterpret_cast<const uint32_t *>(prev) + i0 / EPW;
@@ -179,12 +181,18 @@ __device__ __forceinline__ void unit_combine(const Gen &g, bool first, const voi
                 for (int j = 0; j < NW; ++j) pw[j] = ld_relaxed_u32(p32 + j);
             }
         } else if (DT == SIFAR_BF16) {
+            /* ragged last unit: element loads, all issued before any is used (a loop that tests the bound
+               between loads serialises up to six L2 round trips on the chain's critical path) */
             const uint16_t *p16 = reinterpret_cast<const uint16_t *>(prev);
-            for (int k = 0; k < NW * 2 && i0 + k < n; ++k)
-                pw[k >> 1] |= (uint32_t)ld_relaxed_u16(p16 + i0 + k) << ((k & 1) * 16);
+            uint16_t h[NW * 2];
+#pragma unroll
+            for (int k = 0; k < NW * 2; ++k) h[k] = (i0 + k < n) ? ld_relaxed_u16(p16 + i0 + k) : (uint16_t)0;
+#pragma unroll
+            for (int k = 0; k < NW * 2; ++k) pw[k >> 1] |= (uint32_t)h[k] << ((k & 1) * 16);
         } else {
             const uint32_t *p32 = reinterpret_cast<const uint32_t *>(prev);
-            for (int k = 0; k < NW && i0 + k < n; ++k) pw[k] = ld_relaxed_u32(p32 + i0 + k);
+#pragma unroll
+            for (int k = 0; k < NW; ++k) pw[k] = (i0 + k < n) ? ld_relaxed_u32(p32 + i0 + k) : 0u;
         }
     }
 #pragma unroll
@@ -362,7 +370,7 @@ struct PersistArgs {
     PollShape poll;
     ChainDev *cs;
     ChunkFlags *chunks;
-    unsigned long long *stamps;     /* steps + 1                           */
+    unsigned long long *stamps;     /* C x (steps + 1): per chunk, start of the run and every published result */
     unsigned long long *trace;      /* NULL, or steps x kTraceSlots phase stamps of chunk 0 (see sifar_workload.h) */
     uint32_t *retry_steps;          /* steps: 1 if any CTA re-loaded a slot in that step */
 };
@@ -414,6 +422,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
     const size_t n = (size_t)a.n;
     constexpr int EPU = (MODE == SIFAR_SPECULATIVE) ? ((DT == SIFAR_BF16) ? 6 : 3) : ((DT == SIFAR_BF16) ? 8 : 4);
     const size_t nunits = (n + EPU - 1) / EPU;
+    const size_t n_io = nunits * EPU;         /* ring rows are padded: whole units are read and written */
     const size_t unit0 = (size_t)chunk * kChainThreads * a.K + threadIdx.x;
     __shared__ int s_ok;
     __shared__ int s_retried[2];
@@ -421,8 +430,10 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
     __syncthreads();
     unsigned reloads = 0;
     bool alive = true;
-    const bool stamper = (blockIdx.x == 0);     /* reducer of chunk 0 (or rank 0's producer of chunk 0 without all-reduce) */
-    if (stamper && threadIdx.x == 0) a.stamps[0] = globaltimer_ns();
+    /* the CTA that publishes chunk results stamps them: the chunk's reducer (rank 0's producer without all-reduce) */
+    const bool stamper = no_ar ? (rank == 0u) : is_reducer;
+    unsigned long long *my_stamps = a.stamps + (size_t)chunk * (a.steps + 1u);
+    if (stamper && threadIdx.x == 0) my_stamps[0] = globaltimer_ns();
     /* phase trace: thread 0 of the reducer of chunk 0 and of rank 0's producer of chunk 0 */
     const bool tracer = TRACE && a.trace != nullptr && threadIdx.x == 0 && chunk == 0;
 #define SIFAR_TRACE(slot) do { if (TRACE && tracer) a.trace[(size_t)s * kTraceSlots + (slot)] = globaltimer_ns(); } while (0)
@@ -492,9 +503,9 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                         SIFAR_TRACE(1);
                         if (TRACE && tracer) a.trace[(size_t)s * kTraceSlots + 29] = reloads - before;
                     }
-                    store_slot_result<DT>(ring_row, u, n, sum_vec<DT, P>(x, false));
+                    store_slot_result<DT>(ring_row, u, n_io, sum_vec<DT, P>(x, false));
                 } else {
-                    store_vec_result<DT>(ring_row, u, n, sum_vec<DT, P>(x, true));
+                    store_vec_result<DT>(ring_row, u, n_io, sum_vec<DT, P>(x, true));
                 }
             }
             /* "somebody in this CTA re-loaded a slot": two alternating words, so that clearing one after the
@@ -509,7 +520,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                     s_retried[s & 1u] = 0;
                     st_relaxed_u32(&a.retry_steps[s], 1u);
                 }
-                if (stamper) a.stamps[s + 1u] = globaltimer_ns();
+                if (stamper) my_stamps[s + 1u] = globaltimer_ns();
                 if (MODE == SIFAR_BARRIER_ONESHOT) {
                     /* bottom barrier, reducer side: last CTA to finish reading releases the done flags */
                     const uint32_t arrived = atom_add_acq_rel_u32(&a.cs->bottom_count, 1u) + 1u;
@@ -553,9 +564,11 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                 if (u >= nunits) break;
                 uint32_t w[NW];
                 if (k == 0) {
-                    unit_combine<DT, NW>(g, first, prev, u * EPU, n, z0, w);
+                    unit_combine<DT, NW>(g, first, prev, u * EPU, n, z0, w, no_ar ? 0 : n_io);
                 } else {
-                    produce_words<DT, NW>(g, first, prev, u * EPU, n, w);
+                    float z[NE];
+                    unit_noise<DT, NW>(g, first, u * EPU, n, z);
+                    unit_combine<DT, NW>(g, first, prev, u * EPU, n, z, w, no_ar ? 0 : n_io);
                 }
                 if (MODE == SIFAR_SPECULATIVE) {
                     store_slot(reinterpret_cast<uint4 *>(a.slots + ((size_t)p * P + rank) * a.slot_stride), u,
@@ -575,7 +588,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                 SIFAR_TRACE(6 + 3 * rank);
             } else if (no_ar) {
                 __syncthreads();
-                if (stamper && threadIdx.x == 0) a.stamps[s + 1u] = globaltimer_ns();
+                if (stamper && threadIdx.x == 0) my_stamps[s + 1u] = globaltimer_ns();
             }
         }
     }
@@ -588,14 +601,22 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
     __syncthreads();
     if (threadIdx.x == 0) {
         const uint32_t left = atom_add_acq_rel_u32(&a.cs->exit_count, 1u) + 1u;
-        if (left == a.exit_base + gridDim.x && !no_ar && ld_relaxed_u32(&st->status) == 0u) {
-            unsigned long long with_retry = 0;
-            for (uint32_t s = 0; s < a.steps; ++s) {
-                with_retry += ld_relaxed_u32(&a.retry_steps[s]);
+        s_ok = (left == a.exit_base + gridDim.x && !no_ar && ld_relaxed_u32(&st->status) == 0u);
+    }
+    __syncthreads();
+    if (s_ok) {
+        /* last CTA out: the whole CTA sums and clears the per-step retry marks, then thread 0 books the run */
+        if (MODE == SIFAR_SPECULATIVE) {
+            unsigned long long part = 0;
+            for (uint32_t s = threadIdx.x; s < a.steps; s += kChainThreads) {
+                part += ld_relaxed_u32(&a.retry_steps[s]);
                 st_relaxed_u32(&a.retry_steps[s], 0u);
             }
-            st->stats[kStatCalls] += a.steps;
-            st->stats[kStatCallsWithRetry] += with_retry;
+            if (part) atomicAdd(&st->stats[kStatCallsWithRetry], part);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            atomicAdd(&st->stats[kStatCalls], (unsigned long long)a.steps);
             st_release_u32(&st->epoch, a.e0 + a.steps);
         }
     }
@@ -692,7 +713,9 @@ static bool valid_workload(const sifar_workload *w)
 extern "C" size_t sifar_chain_ring_stride(int dtype, size_t n)
 {
     if (dtype != SIFAR_BF16 && dtype != SIFAR_F32) return 0;
-    return (n * elem_size(dtype) + 255) / 256 * 256;
+    /* room for one whole slot or vector past the last element: the persistent chain reads and writes its
+       ragged last unit in full (sub-sector stores and the loads that follow them are slow at the L2) */
+    return (n * elem_size(dtype) + 16 + 255) / 256 * 256;
 }
 
 template <int DT>
@@ -873,13 +896,13 @@ static int chain_setup_persistent(sifar_chain *ch)
     }
     SIFAR_CUDA(cudaMalloc(&ch->d_cs, sizeof(ChainDev)));
     SIFAR_CUDA(cudaMalloc(&ch->d_chunks, sizeof(ChunkFlags) * C));
-    SIFAR_CUDA(cudaMalloc(&ch->d_stamps, sizeof(unsigned long long) * (ch->steps + 1)));
+    SIFAR_CUDA(cudaMalloc(&ch->d_stamps, sizeof(unsigned long long) * (ch->steps + 1) * C));
     SIFAR_CUDA(cudaMalloc(&ch->d_trace, sizeof(unsigned long long) * ch->steps * kTraceSlots));
     SIFAR_CUDA(cudaMemset(ch->d_trace, 0, sizeof(unsigned long long) * ch->steps * kTraceSlots));
     SIFAR_CUDA(cudaMalloc(&ch->d_retry_steps, sizeof(uint32_t) * ch->steps));
     SIFAR_CUDA(cudaMemset(ch->d_cs, 0, sizeof(ChainDev)));
     SIFAR_CUDA(cudaMemset(ch->d_chunks, 0, sizeof(ChunkFlags) * C));
-    SIFAR_CUDA(cudaMemset(ch->d_stamps, 0, sizeof(unsigned long long) * (ch->steps + 1)));
+    SIFAR_CUDA(cudaMemset(ch->d_stamps, 0, sizeof(unsigned long long) * (ch->steps + 1) * C));
     SIFAR_CUDA(cudaMemset(ch->d_retry_steps, 0, sizeof(uint32_t) * ch->steps));
     return SIFAR_OK;
 }
@@ -1024,9 +1047,36 @@ extern "C" int sifar_chain_stamps(sifar_chain *ch, unsigned long long *stamps)
         return SIFAR_ERR_INVALID;
     }
     SIFAR_CUDA(cudaDeviceSynchronize());
-    SIFAR_CUDA(cudaMemcpy(stamps, ch->d_stamps, sizeof(unsigned long long) * (ch->steps + 1), cudaMemcpyDeviceToHost));
+    const size_t per = (size_t)ch->steps + 1;
+    std::vector<unsigned long long> all(per * ch->C);
+    SIFAR_CUDA(cudaMemcpy(all.data(), ch->d_stamps, sizeof(unsigned long long) * all.size(), cudaMemcpyDeviceToHost));
+    /* a result is complete when its last chunk is: per step the latest stamp over the chunks; the run starts
+       with the earliest CTA */
+    for (size_t s = 0; s < per; ++s) {
+        unsigned long long v = all[s];
+        for (uint32_t c = 1; c < ch->C; ++c) {
+            const unsigned long long x = all[(size_t)c * per + s];
+            v = (s == 0) ? (x < v ? x : v) : (x > v ? x : v);
+        }
+        stamps[s] = v;
+    }
     return SIFAR_OK;
 }
+
+extern "C" int sifar_chain_chunk_stamps(sifar_chain *ch, int chunk, unsigned long long *stamps)
+{
+    if (!ch || !stamps || ch->impl != SIFAR_CHAIN_PERSISTENT || chunk < 0 || (uint32_t)chunk >= ch->C) {
+        set_error("sifar_chain_chunk_stamps: needs a persistent chain, a chunk below %u and a destination", ch ? ch->C : 0u);
+        return SIFAR_ERR_INVALID;
+    }
+    SIFAR_CUDA(cudaDeviceSynchronize());
+    const size_t per = (size_t)ch->steps + 1;
+    SIFAR_CUDA(cudaMemcpy(stamps, ch->d_stamps + (size_t)chunk * per, sizeof(unsigned long long) * per,
+                          cudaMemcpyDeviceToHost));
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_chain_chunks(sifar_chain *ch) { return ch && ch->impl == SIFAR_CHAIN_PERSISTENT ? (int)ch->C : 0; }
 
 extern "C" int sifar_chain_trace(sifar_chain *ch, int enable, unsigned long long *phases)
 {
