@@ -102,14 +102,18 @@ int sifar_chain_chunks(sifar_chain *chain);
 /*
  * Phase timeline of the persistent chain (the latency breakdown that stands in for
  * a bandwidth figure at decode payloads).  enable != 0 makes later runs record,
- * for every step s of a run, 32 %globaltimer stamps (0 = not taken) written by
- * thread 0 of the CTAs that own chunk 0:
- *   reducer:            [0] enters the step      [1] arrival flags seen (speculative: own slot valid)
+ * for every step s of a run, 48 words (0 = not taken; %globaltimer nanoseconds
+ * unless stated) written by the CTAs that own chunk 0:
+ *   reducer, thread 0:  [0] enters the step      [1] arrival flags seen (speculative: its warp's slots valid)
  *                       [2] whole chunk reduced  [3] ready flag released
  *                       [28] done flags released (BARRIER_ONESHOT, last reducer CTA only)
- *   producer of rank r: [4+3r] previous result's ready flag seen   [5+3r] stores issued
- *                       [6+3r] arrival flag released (barrier modes)
- * If `phases` is not NULL the stamps of the last run (steps_per_run x 32) are copied
+ *                       [29] number of slot re-loads of thread 0 in this step (a count)
+ *                       [30..37] end of its first eight re-poll rounds (speculative)
+ *   reducer, lane 0 of warp w:   [38+w] the warp's slots validated (speculative)
+ *   producer of rank r, thread 0: [4+3r] previous result's ready flag seen   [5+3r] stores issued
+ *                                 [6+3r] arrival flag released (barrier modes)
+ *   producer of rank 0, lane 0 of warp w: [42+w] the warp's stores issued
+ * If `phases` is not NULL the words of the last run (steps_per_run x 48) are copied
  * to it (synchronizes the device).  PERSISTENT chains with P = 2 or P = 8 only; the
  * traced kernel is a separate build, so an untraced run pays nothing for it.
  */
