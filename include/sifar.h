@@ -109,6 +109,13 @@ int sifar_destroy(sifar_ctx *ctx);
  * kernel give up: the sticky status becomes SIFAR_ERR_TIMEOUT, `out` is undefined
  * and later calls fail until sifar_reset().  Calls on one context must be
  * enqueued on one stream (or otherwise serialized).
+ *
+ * The early start pays only if the producers can actually run while the reducer
+ * waits.  CUDA does not promise that for independently launched kernels: with
+ * separate streams it held in every measurement here, but inside a captured graph
+ * a waiting reducer of more than about 64 CTAs (n > 98 304 bf16 at P = 8) kept the
+ * producers off the SMs it occupied.  For payloads of that size enqueue the
+ * reducer behind its producers (an event or a graph edge); nothing is lost there.
  */
 int sifar_allreduce(sifar_ctx *ctx, const void *const *rank_ptrs, void *out, size_t n,
                     int mode, void *stream);

@@ -184,6 +184,11 @@ def test_persistent_chain_timestamps_are_monotonic():
             sf.sifar_chain_run(ch, 0)
             stamps = np.array(sf.sifar_chain_stamps(ch, steps), dtype=np.int64)
             assert np.all(np.diff(stamps) >= 0) and stamps[-1] - stamps[0] < 50_000_000
+            # a result is complete with its last chunk: the run's stamps bound every chunk's own stamps
+            C = sf.sifar_chain_chunks(ch)
+            assert C == -(-sf.sifar_slot_count(BF16, n) // 128) if mode == sf.SPECULATIVE else C >= 1
+            per_chunk = np.array([sf.sifar_chain_chunk_stamps(ch, c, steps) for c in range(C)], dtype=np.int64)
+            assert np.array_equal(per_chunk[:, 1:].max(axis=0), stamps[1:]) and per_chunk[:, 0].min() == stamps[0]
             sf.sifar_chain_destroy(ch)
             sf.sifar_reset(ctx.h, 0)
 
