@@ -303,6 +303,31 @@ def payload_sweep(sf, torch, exps=range(10, 26), ranks=(2, 4, 8)):
     return rows
 
 
+def retry_overhead(sf, torch, synth, ranks=(2, 4, 8), kbytes=(8, 16, 32), forced=(0, 1, 2, 3)):
+    """Section 7, "Retry Overhead": p50 per all-reduce of the persistent chain with a fixed number of
+    forced retries, next to the barrier baseline of the same chain."""
+    res = {}
+    for P_ in ranks:
+        for kb in kbytes:
+            n = kb * 1024 // 2
+            row = {}
+            base = Chain(sf, torch, synth, n, sf.BARRIER_ONESHOT, sf.CHAIN_PERSISTENT, ranks=P_)
+            spec = Chain(sf, torch, synth, n, sf.SPECULATIVE, sf.CHAIN_PERSISTENT, ranks=P_)
+            for c in (base, spec):
+                for _ in range(3):
+                    c.run()
+                c.stream.synchronize()
+            row["barrier_oneshot_p50_us"] = round(pct(base.intervals_us(8), 50), 3)
+            for k in forced:
+                sf.sifar_debug_force_retries(spec.ctx, k)
+                spec.run()
+                row[f"speculative_forced{k}_p50_us"] = round(pct(spec.intervals_us(8), 50), 3)
+            base.close()
+            spec.close()
+            res[f"P{P_}_{kb}KB"] = row
+    return res
+
+
 def run_gpu(args) -> None:
     import torch
     from paper_2607_08973_b200 import binding as sf
@@ -355,6 +380,7 @@ def run_gpu(args) -> None:
                 for b in (2, 4, 8, 16)}
             detail["streams"] = measure_modes(sf, torch, synth, n, 3, 8, (sf.CHAIN_STREAMS,), modes, rounds=2)
             detail["payload_sweep"] = payload_sweep(sf, torch)
+            detail["retry_overhead"] = retry_overhead(sf, torch, synth)
         # -- 3. roofline: 16 MiB per rank, inputs larger than L2 -------------------------------------
         r_iters = max(5, min(20, args.steps))
         mean_s, med_s, cnt = measure_roofline(sf, torch, P, LARGE_N, sf.SPECULATIVE, 3, r_iters)

@@ -189,6 +189,19 @@ int sifar_reset(sifar_ctx *ctx, void *stream);
 int sifar_debug_set_epoch(sifar_ctx *ctx, unsigned calls_so_far);
 
 /*
+ * Measurement hook for the retry-latency experiment (Section 7, "Retry Overhead":
+ * latency of the no-retry case and what each further retry adds, obtained by
+ * forcing a fixed number of retries).  With rounds = k > 0 the speculative reducer
+ * treats the attempt that found all P copies of a slot valid as mis-speculated,
+ * k times: it loads all P copies again, one round after another, and validates
+ * the last copies as usual.  Results are unchanged; the statistics count the extra
+ * loads as re-loads and every such call as a call with retry.  rounds <= 64.
+ * Takes effect for sifar_allreduce calls enqueued afterwards, for the next run of
+ * a persistent chain, and for stream / graph chains created afterwards.
+ */
+int sifar_debug_force_retries(sifar_ctx *ctx, unsigned rounds);
+
+/*
  * All-reduce without any allocation.  The paper has no counterpart for this call.
  *
  * For callers that must not allocate device memory: an engine that gave the whole

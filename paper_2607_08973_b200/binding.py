@@ -49,6 +49,7 @@ def lib() -> ctypes.CDLL:
             "sifar_set_timeout_us": (ci, [vp, cu]),
             "sifar_reset": (ci, [vp, vp]),
             "sifar_debug_set_epoch": (ci, [vp, cu]),
+            "sifar_debug_force_retries": (ci, [vp, cu]),
             "sifar_slot_count": (sz, [ci, sz]),
             "sifar_algorithmic_bytes": (sz, [ci, ci, sz, ci]),
             "sifar_last_error": (ctypes.c_char_p, []),
@@ -136,6 +137,10 @@ def sifar_reset(ctx: int, stream: int = 0) -> int:
 
 def sifar_debug_set_epoch(ctx: int, calls_so_far: int) -> int:
     return _check(lib().sifar_debug_set_epoch(ctx, calls_so_far))
+
+
+def sifar_debug_force_retries(ctx: int, rounds: int) -> int:
+    return _check(lib().sifar_debug_force_retries(ctx, rounds))
 
 
 def sifar_slot_count(dtype: int, n: int) -> int:

@@ -307,13 +307,24 @@ __device__ __forceinline__ Roles cta_arrive(const ReduceArgs &a, uint32_t e, int
         } else if (!dead) {
             r.janitor = blockIdx.x + a.janitors - n + 1u;              /* 1 .. G */
             red_add_relaxed_u32(&st->cta_arrive, 1u);
+            /* Janitor 1 re-arms the counter as soon as it has seen it complete with nothing queued; a janitor
+               that polls a moment later would never see it complete.  So the wait also ends when the call
+               has been published, which in this phase only that fast path does. */
             Deadline d;
-            while (ld_acquire_u32(&st->cta_arrive) < n) {
+            bool published = false;
+            for (;;) {
+                const uint32_t count = ld_relaxed_u32(&st->cta_arrive);
+                const uint2 es = ld_relaxed_u32x2(&st->epoch);
+                if (count >= n) break;
+                if (es.x == e) { published = true; break; }
+                if (es.y != 0u) { r.ok = 0u; break; }
                 if (d.expired(a.timeout_ns)) { fail(st, a.host_status, SIFAR_ERR_TIMEOUT); r.ok = 0u; break; }
-                if ((d.polls % 64u) == 0u && ld_relaxed_u32(&st->status) != 0u) { r.ok = 0u; break; }
             }
-            r.ndefer = ld_relaxed_u32(a.defer);
-            if (r.ok && r.ndefer == 0u) {
+            __threadfence();                                           /* the queue entries of the CTAs counted */
+            r.ndefer = published ? 0u : ld_relaxed_u32(a.defer);
+            if (published) {
+                r.janitor = 0u;
+            } else if (r.ok && r.ndefer == 0u) {
                 /* Nothing was queued (the usual case): janitor 1 publishes at once, the others just leave. */
                 if (r.janitor == 1u) {
                     st_relaxed_u32(&st->cta_arrive, 0u);
@@ -613,6 +624,7 @@ sifar::PollShape sifar::poll_shape_for(const sifar_ctx *ctx, size_t n)
     p.wide = pairs <= ctx->poll_wide_max ? 1u : 0u;
     p.pace_ns = pairs <= ctx->poll_pace_min ? 0u : ctx->poll_pace_ns;
     p.sentinel = pairs <= ctx->poll_sentinel_min ? 0u : 1u;
+    p.forced = ctx->force_retries;
     return p;
 }
 
@@ -1001,6 +1013,14 @@ extern "C" int sifar_debug_set_epoch(sifar_ctx *c, unsigned calls_so_far)
     SIFAR_CUDA(cudaDeviceSynchronize());
     c->h_epoch = calls_so_far;
     c->last_mode0_epoch = 0;
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_debug_force_retries(sifar_ctx *c, unsigned rounds)
+{
+    if (!c) { set_error("sifar_debug_force_retries: NULL context"); return SIFAR_ERR_INVALID; }
+    if (rounds > 64u) { set_error("sifar_debug_force_retries: at most 64 rounds"); return SIFAR_ERR_INVALID; }
+    c->force_retries = rounds;
     return SIFAR_OK;
 }
 

@@ -88,6 +88,7 @@ struct sifar_ctx {
     size_t poll_pace_min;            /* ... paced polling above this many pairs                              */
     uint32_t poll_pace_ns;
     size_t poll_sentinel_min;        /* ... sentinel wait per warp above this many pairs (persistent chain) */
+    uint32_t force_retries;          /* measurement knob: forced re-load rounds per slot (0 in normal use)    */
     /* staging for sifar_allreduce_host, allocated on first use */
     char *d_stage_in;
     char *d_stage_out;

@@ -146,6 +146,7 @@ struct PollShape {
     uint32_t wide;
     uint32_t pace_ns;
     uint32_t sentinel;     /* wait on one slot per rank and warp before touching the warp's other slots */
+    uint32_t forced;       /* measurement knob: re-load every slot this many times although it may be valid */
 };
 
 /*
@@ -178,9 +179,9 @@ __device__ __forceinline__ bool sentinel_wait(const uint4 *const *src, size_t wa
 }
 
 template <int P>
-__device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const *src, size_t s, uint32_t e,
+__device__ __forceinline__ bool validate_once(uint4 (&x)[P], const uint4 *const *src, size_t s, uint32_t e,
                                               unsigned long long timeout_ns, PollShape shape, unsigned &reloads,
-                                              unsigned long long *round_stamps = nullptr)
+                                              unsigned long long *round_stamps)
 {
     uint32_t stale = 0;
 #pragma unroll
@@ -188,6 +189,30 @@ __device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const 
     if (stale == 0u) return true;
     return shape.wide ? revalidate<P, true>(x, stale, src, s, e, timeout_ns, shape.pace_ns, reloads, round_stamps)
                       : revalidate<P, false>(x, stale, src, s, e, timeout_ns, shape.pace_ns, reloads, round_stamps);
+}
+
+template <int P>
+__device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const *src, size_t s, uint32_t e,
+                                              unsigned long long timeout_ns, PollShape shape, unsigned &reloads,
+                                              unsigned long long *round_stamps = nullptr)
+{
+    if (!validate_once<P>(x, src, s, e, timeout_ns, shape, reloads, round_stamps)) return false;
+    if (shape.forced == 0u) return true;
+    /* Forced retries (the retry-latency experiment of Section 7, "Retry Overhead"): the attempt that found
+       every copy valid is treated as mis-speculated, `forced` times: each round loads all P copies again.
+       The address of a round depends on the previous round's tags through a zero the compiler cannot see,
+       so the rounds run one after another as real retries do.  The last copies are validated as usual
+       (a valid slot stays valid until its producer's store for call e + 2, which waits for this result). */
+    for (uint32_t k = 0; k < shape.forced; ++k) {
+        uint32_t dep = 0;
+#pragma unroll
+        for (int r = 0; r < P; ++r) dep |= x[r].w;
+        asm volatile("and.b32 %0, %0, 0;" : "+r"(dep));
+#pragma unroll
+        for (int r = 0; r < P; ++r) x[r] = ld_slot(src[r] + s + dep);
+        reloads += P;
+    }
+    return validate_once<P>(x, src, s, e, timeout_ns, shape, reloads, nullptr);
 }
 
 /* ------------------------------------------------------------------------ */
