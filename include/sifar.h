@@ -27,6 +27,10 @@
  *   SIFAR_POLL_PACE_NS/_MIN sleep between polling rounds above _MIN pairs (0 = unpaced)
  *   SIFAR_POLL_SENTINEL_MIN persistent chain: above this many pairs a warp first waits on one slot per rank (16384)
  *   SIFAR_CHAIN_CLUSTER     0 = persistent chain without thread-block clusters
+ *   SIFAR_PDL               0 = reducers are launched without programmatic dependent launch (read when the
+ *                           library is loaded).  By default a reducer with more CTAs than the GPU has SMs
+ *                           may become resident while the kernel before it on its stream drains; it reads
+ *                           nothing until that kernel is complete.
  *
  * All pointers named "device" are CUDA device pointers valid on the context's
  * device; "stream" arguments are cudaStream_t passed as void* (NULL = the legacy

@@ -313,14 +313,13 @@ __device__ __forceinline__ Roles cta_arrive(const ReduceArgs &a, uint32_t e, int
             Deadline d;
             bool published = false;
             for (;;) {
-                const uint32_t count = ld_relaxed_u32(&st->cta_arrive);
-                const uint2 es = ld_relaxed_u32x2(&st->epoch);
+                const uint2 es = ld_relaxed_u32x2(&st->epoch);         /* issued first: not held back by the acquire */
+                const uint32_t count = ld_acquire_u32(&st->cta_arrive); /* acquire: the queue entries of the CTAs counted */
                 if (count >= n) break;
                 if (es.x == e) { published = true; break; }
                 if (es.y != 0u) { r.ok = 0u; break; }
                 if (d.expired(a.timeout_ns)) { fail(st, a.host_status, SIFAR_ERR_TIMEOUT); r.ok = 0u; break; }
             }
-            __threadfence();                                           /* the queue entries of the CTAs counted */
             r.ndefer = published ? 0u : ld_relaxed_u32(a.defer);
             if (published) {
                 r.janitor = 0u;
@@ -374,6 +373,10 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a
     constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
     const size_t ntiles = tiles_for((size_t)a.n / EPV, U);
     const size_t tile = blockIdx.x;
+    /* programmatic dependent launch: nothing is read before the previous kernel of the stream is complete;
+       the next kernel may become resident as soon as every CTA of this one has started */
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
     int give_up = 0;
     uint32_t e = top_barrier<P>(a, a.two_phase ? a.spin_ns : a.timeout_ns, give_up);
     bool alive = true;
@@ -413,6 +416,9 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
     const size_t tile = blockIdx.x;
     const unsigned long long limit_ns = a.two_phase ? a.spin_ns : a.timeout_ns;
     unsigned reloads = 0;
+    /* programmatic dependent launch, as in k_reduce_plain */
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
 
     /* The call number is loaded together with the slots (no dependent round trip before the data), by one
        thread per CTA: a word that every warp of a large grid loads becomes a hot spot in its L2 slice. */
@@ -469,6 +475,8 @@ __device__ __forceinline__ void pack_body(const PackArgs &a)
 {
     DevState *st = a.st;
     __shared__ uint32_t s_epoch;
+    /* a reducer that follows on the same stream may become resident now; it waits for this grid's completion */
+    asm volatile("griddepcontrol.launch_dependents;");
     if (threadIdx.x == 0) {
         const uint2 es = ld_relaxed_u32x2(&st->epoch);
         uint32_t e = es.x + 1u;
@@ -588,15 +596,37 @@ __global__ void k_set_epoch(DevState *st, uint32_t e) { st->epoch = e; }
 /* ------------------------------------------------------------------------ */
 /* launch geometry                                                           */
 /* ------------------------------------------------------------------------ */
+/*
+ * Programmatic dependent launch: a reducer may become resident while the kernel before it on its stream
+ * is still draining.  Its CTAs then sit in griddepcontrol.wait until that kernel has completed and its
+ * writes are visible, so what they read is unchanged; what is saved is the launch gap and the ramp-up
+ * between back-to-back kernels (about 2 us per pair).  Used for reducer grids above the SM count, where
+ * bandwidth is what counts.  SIFAR_PDL=0 launches the plain way.
+ */
+static bool g_pdl = !(getenv("SIFAR_PDL") && atoi(getenv("SIFAR_PDL")) == 0);
+
+template <typename K>
+static cudaError_t launch_k(K kernel, int grid, cudaStream_t s, const ReduceArgs &a)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(kThreads); cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    /* only for grids above the SM count: at decode payloads the early-resident reducer measurably slows
+       the graph chains and the host path (its blocked CTAs sit beside the kernels it waits for) */
+    cfg.attrs = at; cfg.numAttrs = (g_pdl && a.two_phase) ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
 template <int DT, int P>
 static cudaError_t launch_reduce_p(int mode, int grid, cudaStream_t s, const ReduceArgs &a)
 {
     switch (mode) {
-    case SIFAR_BARRIER_ONESHOT: k_reduce_plain<DT, P, SIFAR_BARRIER_ONESHOT><<<grid, kThreads, 0, s>>>(a); break;
-    case SIFAR_DUALBUF:         k_reduce_plain<DT, P, SIFAR_DUALBUF><<<grid, kThreads, 0, s>>>(a); break;
-    default:                    k_reduce_spec<DT, P><<<grid, kThreads, 0, s>>>(a); break;
+    case SIFAR_BARRIER_ONESHOT: return launch_k(k_reduce_plain<DT, P, SIFAR_BARRIER_ONESHOT>, grid, s, a);
+    case SIFAR_DUALBUF:         return launch_k(k_reduce_plain<DT, P, SIFAR_DUALBUF>, grid, s, a);
+    default:                    return launch_k(k_reduce_spec<DT, P>, grid, s, a);
     }
-    return cudaGetLastError();
 }
 
 template <int DT>
