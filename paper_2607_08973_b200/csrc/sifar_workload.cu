@@ -376,6 +376,7 @@ struct PersistArgs {
 };
 
 constexpr int kChainThreads = 128;
+constexpr int kPreUnits = 4;            /* units per producer thread, beyond its first, whose seeded half is computed before the wait */
 constexpr int kTraceSlots = 48;         /* 0-3 reducer, 4 + 3r .. 6 + 3r rank r's producer, 28 done flags */
 
 /* Bounded wait that also gives up when another CTA has already recorded a failure. */
@@ -393,7 +394,7 @@ __device__ __forceinline__ bool chain_wait(const uint32_t *flag, uint32_t want, 
 }
 
 template <int DT, int P, int MODE, bool TRACE>
-__global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
+__global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
 {
     DevState *st = a.st;
     const uint32_t C = a.C;
@@ -426,6 +427,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
     const size_t unit0 = (size_t)chunk * kChainThreads * a.K + threadIdx.x;
     __shared__ int s_ok;
     __shared__ int s_retried[2];
+    __shared__ float s_z[kPreUnits][8][kChainThreads];   /* producers: seeded halves computed ahead of the wait */
     if (threadIdx.x < 2) s_retried[threadIdx.x] = 0;
     __syncthreads();
     unsigned reloads = 0;
@@ -535,14 +537,24 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
             constexpr int NE = NW * ((DT == SIFAR_BF16) ? 2 : 1);
             const Gen g = make_gen(a.w, rank, t);
             const bool first = (t == 1u);
-            /* the seeded half of the first unit does not need the previous result: do it before waiting */
+            /* the seeded half of a unit does not need the previous result: do it before waiting.  The first
+               unit's stays in registers, those of the next kPreUnits units are parked in shared memory (grids
+               that need more units per thread than that are far beyond the decode payloads) */
             float z0[NE];
-            const bool pre = (unit0 < nunits);
-            if (pre) {
+            if (unit0 < nunits) {
                 unit_noise<DT, NW>(g, first, unit0 * EPU, n, z0);
                 /* pin the values here: without this the compiler sinks the arithmetic below the wait */
 #pragma unroll
                 for (int k = 0; k < NE; ++k) asm volatile("" : "+f"(z0[k]));
+            }
+#pragma unroll 1
+            for (uint32_t k = 1; k < a.K && k <= (uint32_t)kPreUnits; ++k) {
+                const size_t u = unit0 + (size_t)k * kChainThreads;
+                if (u >= nunits) break;
+                float z[NE];
+                unit_noise<DT, NW>(g, first, u * EPU, n, z);
+#pragma unroll
+                for (int q = 0; q < NE; ++q) s_z[k - 1u][q][threadIdx.x] = z[q];
             }
             if (threadIdx.x == 0) {
                 bool ok = true;
@@ -559,17 +571,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
             if (!s_ok) { alive = false; break; }
             const char *prev = no_ar ? a.plain + ((size_t)(p ^ 1u) * P + rank) * a.plain_stride
                                      : a.ring + (size_t)((t + a.ring_len - 2u) % a.ring_len) * a.ring_stride;
-            for (uint32_t k = 0; k < a.K; ++k) {
-                const size_t u = unit0 + (size_t)k * kChainThreads;
-                if (u >= nunits) break;
-                uint32_t w[NW];
-                if (k == 0) {
-                    unit_combine<DT, NW>(g, first, prev, u * EPU, n, z0, w, no_ar ? 0 : n_io);
-                } else {
-                    float z[NE];
-                    unit_noise<DT, NW>(g, first, u * EPU, n, z);
-                    unit_combine<DT, NW>(g, first, prev, u * EPU, n, z, w, no_ar ? 0 : n_io);
-                }
+            const auto store_unit = [&](size_t u, const uint32_t (&w)[NW]) {
                 if (MODE == SIFAR_SPECULATIVE) {
                     store_slot(reinterpret_cast<uint4 *>(a.slots + ((size_t)p * P + rank) * a.slot_stride), u,
                                w[0], w[1], w[2], e);
@@ -578,6 +580,26 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(const PersistArgs a)
                     st_slot(reinterpret_cast<uint4 *>(a.plain + ((size_t)bp * P + rank) * a.plain_stride) + u,
                             make_uint4(w[0], w[1], w[2], w[NW - 1]));
                 }
+            };
+            if (unit0 < nunits) {
+                uint32_t w[NW];
+                unit_combine<DT, NW>(g, first, prev, unit0 * EPU, n, z0, w, no_ar ? 0 : n_io);
+                store_unit(unit0, w);
+            }
+#pragma unroll 1
+            for (uint32_t k = 1; k < a.K; ++k) {
+                const size_t u = unit0 + (size_t)k * kChainThreads;
+                if (u >= nunits) break;
+                uint32_t w[NW];
+                float z[NE];
+                if (k <= (uint32_t)kPreUnits) {
+#pragma unroll
+                    for (int q = 0; q < NE; ++q) z[q] = s_z[k - 1u][q][threadIdx.x];
+                } else {
+                    unit_noise<DT, NW>(g, first, u * EPU, n, z);
+                }
+                unit_combine<DT, NW>(g, first, prev, u * EPU, n, z, w, no_ar ? 0 : n_io);
+                store_unit(u, w);
             }
             if (TRACE && a.trace != nullptr && chunk == 0 && rank == 0 && (threadIdx.x & 31) == 0)
                 a.trace[(size_t)s * kTraceSlots + 42 + (threadIdx.x >> 5)] = globaltimer_ns();
@@ -862,8 +884,9 @@ static int chain_setup_persistent(sifar_chain *ch)
     int per_sm = 0;
     SIFAR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, chain_kernel(ch), kChainThreads, 0));
     const size_t resident = (size_t)per_sm * c->sm_count;
-    /* leave half of the machine free: the chain stands for a few operators of a forward pass, not all of it */
-    const size_t budget = resident / 2 > (size_t)roles ? resident / 2 : (size_t)roles;
+    /* the whole machine if need be: every unit per thread beyond the first lengthens the step by its
+       dependent load and store round trips */
+    const size_t budget = resident > (size_t)roles ? resident : (size_t)roles;
     uint32_t K = 1;      /* units per thread and step: 1 whenever the grid fits (more only lengthens the step) */
     size_t C = (units + kChainThreads - 1) / kChainThreads;
     while (C * roles > budget) {
