@@ -125,6 +125,45 @@ int sifar_chain_launches_per_run(sifar_chain *chain);
 int sifar_chain_destroy(sifar_chain *chain);
 
 /*
+ * The same decode step with P readers: every emulated rank runs its own next
+ * operation AND its own pull-and-reduce, as every GPU does in the paper's system
+ * (Section 3.1; the oneshot pseudocode of Section 4.2), and keeps its own copy of
+ * every result.  One cooperative kernel of P x C CTAs; CTA (r, c) computes chunk c
+ * of rank r's partial from chunk c of rank r's copy of the previous result, stores
+ * it, pulls chunk c of all P partials (its own included) and reduces it.  Ranks
+ * are ordered against each other by the mode's protocol alone (P x P arrival and
+ * done flags, or slot tags), so they drift as real GPUs do and a rank
+ * mis-speculates exactly when a peer is behind it.  Results are those of the
+ * one-reader chains, P times.
+ *   out_rings      device, P x ring_len rows of sifar_chain_ring_stride() bytes, caller-owned;
+ *                  rank r's copy of out^t lands in row r * ring_len + (t-1) mod ring_len
+ *   other arguments as for sifar_chain_create (mode may be SIFAR_CHAIN_NO_ALLREDUCE: every rank's
+ *   operation feeds on its own partial, the timing floor)
+ * The chain owns the context exclusively until it is destroyed.
+ */
+typedef struct sifar_symchain sifar_symchain;   /* opaque */
+
+sifar_symchain *sifar_symchain_create(sifar_ctx *ctx, const sifar_workload *w, size_t n, int mode,
+                                      void *out_rings, int ring_len, int steps_per_run);
+/* Enqueue the next steps_per_run steps on `stream`. */
+int sifar_symchain_run(sifar_symchain *chain, void *stream);
+/*
+ * Device timestamps of the last run (synchronizes): stamps[0] = start of the run,
+ * stamps[s] = result s complete on every rank (latest chunk of the latest rank),
+ * s = 1..steps_per_run; sifar_symchain_rank_stamps: the same for one rank's copy.
+ */
+int sifar_symchain_stamps(sifar_symchain *chain, unsigned long long *stamps);
+int sifar_symchain_rank_stamps(sifar_symchain *chain, int rank, unsigned long long *stamps);
+/*
+ * Mis-speculation per rank (Section 7: the fraction of all-reduces that retried):
+ * host_per_rank[r] = number of steps so far in which rank r had to load a slot
+ * again, r = 0..P-1 (speculative mode; zeros otherwise).  Synchronizes.  The
+ * context's statistics count a step as a call with retry if any rank retried.
+ */
+int sifar_symchain_retries(sifar_symchain *chain, unsigned long long *host_per_rank);
+int sifar_symchain_destroy(sifar_symchain *chain);
+
+/*
  * Generator probes (for tests and for building inputs on the device): write the
  * first partial of `rank`, or its partial of step t >= 2 from prev_out, as n plain
  * elements of `dtype` to dst (device, 16-byte aligned).

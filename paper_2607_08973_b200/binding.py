@@ -198,6 +198,12 @@ def _wl() -> ctypes.CDLL:
             "sifar_chain_launches_per_run": (ci, [vp]),
             "sifar_chain_trace": (ci, [vp, ci, ullp]),
             "sifar_chain_destroy": (ci, [vp]),
+            "sifar_symchain_create": (vp, [vp, wp, sz, ci, vp, ci, ci]),
+            "sifar_symchain_run": (ci, [vp, vp]),
+            "sifar_symchain_stamps": (ci, [vp, ullp]),
+            "sifar_symchain_rank_stamps": (ci, [vp, ci, ullp]),
+            "sifar_symchain_retries": (ci, [vp, ullp]),
+            "sifar_symchain_destroy": (ci, [vp]),
             "sifar_workload_first": (ci, [wp, ci, ci, vp, sz, vp]),
             "sifar_workload_next": (ci, [wp, ci, cu, ci, vp, vp, sz, vp]),
             "sifar_workload_delays": (ci, [wp, ci, cu, ctypes.POINTER(cu)]),
@@ -259,6 +265,40 @@ def sifar_chain_launches_per_run(chain: int) -> int:
 
 def sifar_chain_destroy(chain: int) -> int:
     return _check(_wl().sifar_chain_destroy(chain))
+
+
+def sifar_symchain_create(ctx: int, w: sifar_workload, n: int, mode: int, out_rings: int, ring_len: int,
+                          steps_per_run: int) -> int:
+    h = _wl().sifar_symchain_create(ctx, ctypes.byref(w), n, mode, out_rings, ring_len, steps_per_run)
+    if not h:
+        raise SifarError(ERR_INVALID, sifar_last_error())
+    return h
+
+
+def sifar_symchain_run(chain: int, stream: int = 0) -> int:
+    return _check(_wl().sifar_symchain_run(chain, stream))
+
+
+def sifar_symchain_stamps(chain: int, steps_per_run: int) -> list[int]:
+    buf = (ctypes.c_ulonglong * (steps_per_run + 1))()
+    _check(_wl().sifar_symchain_stamps(chain, buf))
+    return list(buf)
+
+
+def sifar_symchain_rank_stamps(chain: int, rank: int, steps_per_run: int) -> list[int]:
+    buf = (ctypes.c_ulonglong * (steps_per_run + 1))()
+    _check(_wl().sifar_symchain_rank_stamps(chain, rank, buf))
+    return list(buf)
+
+
+def sifar_symchain_retries(chain: int, P: int) -> list[int]:
+    buf = (ctypes.c_ulonglong * P)()
+    _check(_wl().sifar_symchain_retries(chain, buf))
+    return list(buf)
+
+
+def sifar_symchain_destroy(chain: int) -> int:
+    return _check(_wl().sifar_symchain_destroy(chain))
 
 
 def sifar_workload_first(w: sifar_workload, rank: int, dtype: int, dst: int, n: int, stream: int = 0) -> int:
