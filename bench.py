@@ -303,6 +303,35 @@ def payload_sweep(sf, torch, exps=range(10, 26), ranks=(2, 4, 8)):
     return rows
 
 
+def measure_symmetric(sf, torch, synth, ranks, n, name="llama", steps=ARS_PER_STEP, warm=3, runs=8):
+    """The chain with P readers (every rank reduces for itself): p50 / p99 us between complete results on all
+    ranks, every mode and the floor without all-reduce; mis-speculation per rank for the speculative mode."""
+    d = synth.chain_workload(name, ranks)
+    res = {}
+    for mode in (sf.BARRIER_ONESHOT, sf.DUALBUF, sf.SPECULATIVE, sf.CHAIN_NO_ALLREDUCE):
+        ctx = sf.sifar_create(ranks, n, 0)
+        stride = sf.sifar_chain_ring_stride(0, n)
+        rings = torch.zeros(ranks * 2 * stride, dtype=torch.uint8, device="cuda")
+        ch = sf.sifar_symchain_create(ctx, sf.make_workload(**d), n, mode, rings.data_ptr(), 2, steps)
+        iv = []
+        for i in range(warm + runs):
+            sf.sifar_symchain_run(ch, 0)
+            if i >= warm:
+                st = np.array(sf.sifar_symchain_stamps(ch, steps), dtype=np.int64)
+                iv.append(np.diff(st)[1:] * 1e-3)
+        iv = np.concatenate(iv)
+        r = {"p50_us": round(pct(iv, 50), 3), "p99_us": round(pct(iv, 99), 3)}
+        if mode == sf.SPECULATIVE:
+            rt = sf.sifar_symchain_retries(ch, ranks)
+            stt = sf.sifar_get_stats(ctx)
+            r["misspeculated_steps_per_rank"] = [round(x / ((warm + runs) * steps), 3) for x in rt]
+            r["slot_reloads_per_call"] = round(stt["slot_reloads"] / max(1, stt["calls"]), 1)
+        res[sf.MODE_NAMES.get(mode, "no_allreduce")] = r
+        sf.sifar_symchain_destroy(ch)
+        sf.sifar_destroy(ctx)
+    return res
+
+
 def retry_overhead(sf, torch, synth, ranks=(2, 4, 8), kbytes=(8, 16, 32), forced=(0, 1, 2, 3)):
     """Section 7, "Retry Overhead": p50 per all-reduce of the persistent chain with a fixed number of
     forced retries, next to the barrier baseline of the same chain."""
@@ -373,7 +402,14 @@ def run_gpu(args) -> None:
         impls = (sf.CHAIN_PERSISTENT,) if args.skip_graph else (sf.CHAIN_PERSISTENT, sf.CHAIN_GRAPH)
         if args.only == "all":
             detail["modes"] = measure_modes(sf, torch, synth, n, args.warmup, max(8, args.steps // 8), impls, modes)
+        if args.only == "all":
+            detail["p_readers"] = {"llama P=8 8KB": measure_symmetric(sf, torch, synth, P, n)}
         if args.sweep and args.only == "all":
+            for P_ in (2, 4, 8):
+                for kb in (8, 16, 32):
+                    if (P_, kb) != (8, 8):
+                        detail["p_readers"][f"llama P={P_} {kb}KB"] = measure_symmetric(sf, torch, synth, P_, kb * 512)
+                detail["p_readers"][f"skew P={P_} 32KB"] = measure_symmetric(sf, torch, synth, P_, 16384, name="skew", runs=4)
             detail["by_batch_tokens"] = {
                 str(b): measure_modes(sf, torch, synth, HIDDEN * b, args.warmup, max(8, args.steps // 8),
                                       (sf.CHAIN_PERSISTENT, sf.CHAIN_GRAPH), modes)
