@@ -43,6 +43,36 @@ def test_config5_ten_thousand_skewed_steps(skew_reference, impl, mode):
         assert 0 < st["calls_with_retry"] <= steps * runs and st["slot_reloads"] > 0
 
 
+@pytest.mark.parametrize("mode", [sf.SPECULATIVE, sf.BARRIER_ONESHOT])
+def test_config5_ten_thousand_skewed_steps_with_p_readers(skew_reference, mode):
+    """The same 10 000 steps with every rank reducing for itself: all eight copies, every step."""
+    d, want = skew_reference
+    P, n, steps, runs = 8, 16384, 100, 100
+    stride = sf.sifar_chain_ring_stride(BF16, n)
+    with Ctx(P, n, BF16, timeout_us=5_000_000) as ctx:
+        rings = torch.zeros(P * steps * stride, dtype=torch.uint8, device="cuda")
+        ch = sf.sifar_symchain_create(ctx.h, sf.make_workload(**d), n, mode, rings.data_ptr(), steps, steps)
+        try:
+            for k in range(runs):
+                sf.sifar_symchain_run(ch, 0)
+                torch.cuda.synchronize()
+                assert sf.sifar_status(ctx.h) == 0
+                h = rings.cpu().numpy().reshape(P, steps, stride)[:, :, : n * 2].view(np.uint16)
+                for r in range(P):
+                    assert np.array_equal(h[r], want[k * steps:(k + 1) * steps]), f"segment {k} rank {r}"
+            st = sf.sifar_get_stats(ctx.h)
+            retries = sf.sifar_symchain_retries(ch, P)
+        finally:
+            sf.sifar_symchain_destroy(ch)
+    assert st["calls"] == steps * runs and st["timeouts"] == 0
+    if mode == sf.SPECULATIVE:
+        # every rank but the last one of a step finds a peer missing: (P-1)/P of the steps on average
+        share = np.array(retries) / (steps * runs)
+        assert np.all(share > 0.7) and np.all(share < 0.98), share
+    else:
+        assert sum(retries) == 0
+
+
 @pytest.mark.parametrize("dtype", [BF16, F32])
 def test_config4_largest_payload_every_mode(oracle, dtype):
     """P=8, n=32 Mi (64 MiB of bf16 / 128 MiB of fp32 per rank): the whole output against the oracle."""
