@@ -254,12 +254,17 @@ struct Roles {
     uint32_t ok;
 };
 
+constexpr uint32_t kQueuedBit = 0x80000000u;
+
 /* Thread 0 of a CTA in the deferring regime: queue the CTA's tile (made visible before the CTA's arrival). */
 __device__ __forceinline__ void defer_tile(const ReduceArgs &a, size_t tile)
 {
     const uint32_t slot = atomicAdd(a.defer, 1u);
     st_relaxed_u32(a.defer + 1u + slot, (uint32_t)tile);
     __threadfence();
+    /* "something is queued" travels in the top bit of the arrival count, set before this thread counts its
+       CTA: who sees the count complete knows from the same word whether the queue needs a look */
+    asm volatile("red.relaxed.gpu.global.or.b32 [%0], %1;" :: "l"(&a.st->cta_arrive), "r"(kQueuedBit) : "memory");
 }
 
 /*
@@ -311,16 +316,17 @@ __device__ __forceinline__ Roles cta_arrive(const ReduceArgs &a, uint32_t e, int
                that polls a moment later would never see it complete.  So the wait also ends when the call
                has been published, which in this phase only that fast path does. */
             Deadline d;
-            bool published = false;
+            bool published = false, queued = false;
             for (;;) {
                 const uint2 es = ld_relaxed_u32x2(&st->epoch);         /* issued first: not held back by the acquire */
                 const uint32_t count = ld_acquire_u32(&st->cta_arrive); /* acquire: the queue entries of the CTAs counted */
-                if (count >= n) break;
+                queued = (count & kQueuedBit) != 0u;
+                if ((count & ~kQueuedBit) >= n) break;
                 if (es.x == e) { published = true; break; }
                 if (es.y != 0u) { r.ok = 0u; break; }
                 if (d.expired(a.timeout_ns)) { fail(st, a.host_status, SIFAR_ERR_TIMEOUT); r.ok = 0u; break; }
             }
-            r.ndefer = published ? 0u : ld_relaxed_u32(a.defer);
+            r.ndefer = (published || !queued) ? 0u : ld_relaxed_u32(a.defer);
             if (published) {
                 r.janitor = 0u;
             } else if (r.ok && r.ndefer == 0u) {
