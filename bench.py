@@ -375,7 +375,7 @@ def run_gpu(args) -> None:
     # -- 1. the timed region: exactly K decode steps, persistent chain, speculative ------------------
     secs, p50, p99, launches = 0.0, 0.0, 0.0, 0
     stats = {"calls": 0, "calls_with_retry": 0, "slot_reloads": 0}
-    if args.only != "roofline":
+    if args.only not in ("roofline", "p_readers"):
         main = Chain(sf, torch, synth, n, sf.SPECULATIVE, sf.CHAIN_PERSISTENT)
         for _ in range(args.warmup):
             main.run()
@@ -395,7 +395,10 @@ def run_gpu(args) -> None:
         main.close()
 
     detail, roof, roof_decode, e2e, cpu = {}, None, None, None, None
-    if rank == 0 and args.only != "decode":
+    if rank == 0 and args.only == "p_readers":
+        detail["p_readers"] = {"llama P=8 8KB": measure_symmetric(sf, torch, synth, P, n, warm=args.warmup,
+                                                                 runs=max(1, args.steps))}
+    if rank == 0 and args.only not in ("decode", "p_readers"):
         # -- 2. every mode and chain implementation on the same step, interleaved -------------------
         w0 = time.time()
         modes = (sf.BARRIER_ONESHOT, sf.DUALBUF, sf.SPECULATIVE, sf.CHAIN_NO_ALLREDUCE)
@@ -506,8 +509,9 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="sifar", choices=["sifar", "reference"])
     ap.add_argument("--sweep", action="store_true", help="also batch sizes 2..16 and the stream chain")
-    ap.add_argument("--only", default="all", choices=["all", "decode", "roofline"],
-                    help="profiling aid: run the timed decode region only, or the roofline section only")
+    ap.add_argument("--only", default="all", choices=["all", "decode", "roofline", "p_readers"],
+                    help="profiling aid: run the timed decode region only, the roofline section only, or the "
+                         "P-reader chain only")
     ap.add_argument("--skip-graph", action="store_true",
                     help="profiling aid: leave out the graph / stream chains (under ncu kernels are serialised, and "
                          "those chains' reducers wait for producers that run concurrently)")
