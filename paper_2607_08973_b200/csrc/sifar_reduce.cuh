@@ -53,6 +53,23 @@ __device__ __forceinline__ int wait_flag_ge(const uint32_t *flag, uint32_t base,
     return (int)d.polls;
 }
 
+/*
+ * Bounded acquire wait of the persistent kernels: until the flag equals (or, GE, has reached) `want`.  Records
+ * SIFAR_ERR_TIMEOUT when the limit passes, and also gives up when another CTA has already recorded a failure.
+ */
+template <bool GE>
+__device__ __forceinline__ bool wait_flag_or_fail(const uint32_t *flag, uint32_t want, DevState *st, int *host_status,
+                                                  unsigned long long timeout_ns)
+{
+    Deadline d;
+    for (;;) {
+        const uint32_t v = ld_acquire_u32(flag);
+        if (GE ? (v >= want) : (v == want)) return true;
+        if (d.expired(timeout_ns)) { fail(st, host_status, SIFAR_ERR_TIMEOUT); return false; }
+        if ((d.polls % 64u) == 0u && ld_relaxed_u32(&st->status) != 0u) return false;
+    }
+}
+
 /* ------------------------------------------------------------------------ */
 /* rank-order accumulation                                                   */
 /* ------------------------------------------------------------------------ */

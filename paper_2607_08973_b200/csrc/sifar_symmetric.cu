@@ -80,20 +80,6 @@ struct SymArgs {
     unsigned long long *rank_retries; /* [P] cumulative (rank, step) pairs with a re-load */
 };
 
-/* Bounded acquire wait that also gives up when another CTA has recorded a failure. */
-template <bool GE>
-__device__ __forceinline__ bool sym_wait(const uint32_t *flag, uint32_t want, DevState *st, int *host_status,
-                                         unsigned long long timeout_ns)
-{
-    Deadline d;
-    for (;;) {
-        const uint32_t v = ld_acquire_u32(flag);
-        if (GE ? (v >= want) : (v == want)) return true;
-        if (d.expired(timeout_ns)) { fail(st, host_status, SIFAR_ERR_TIMEOUT); return false; }
-        if ((d.polls % 64u) == 0u && ld_relaxed_u32(&st->status) != 0u) return false;
-    }
-}
-
 template <int DT, int P, int MODE>
 __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
 {
@@ -141,7 +127,7 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
                 bool ok = true;
                 /* bottom barrier, writer side: all P readers are done with the single buffer (Section 3.1, phase 3) */
                 if (MODE == SIFAR_BARRIER_ONESHOT && !first && threadIdx.x < P)
-                    ok = sym_wait<true>(&cf->done[threadIdx.x], e - 1u, st, a.host_status, a.timeout_ns);
+                    ok = wait_flag_or_fail<true>(&cf->done[threadIdx.x], e - 1u, st, a.host_status, a.timeout_ns);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (threadIdx.x == 0) {
                     if (ok) spin_ns(gen_delay_ns(a.w, rank, t));          /* seeded skew between the ranks */
@@ -189,7 +175,7 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
             if (threadIdx.x < 32) {
                 bool ok = true;
                 if (threadIdx.x < P)
-                    ok = sym_wait<false>(&cf->arrive[p][threadIdx.x], e, st, a.host_status, a.timeout_ns);
+                    ok = wait_flag_or_fail<false>(&cf->arrive[p][threadIdx.x], e, st, a.host_status, a.timeout_ns);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (threadIdx.x == 0) s_ok = ok;
             }

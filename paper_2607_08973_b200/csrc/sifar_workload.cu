@@ -181,20 +181,6 @@ constexpr int kChainThreads = 128;
 constexpr int kPreUnits = 4;            /* units per producer thread, beyond its first, whose seeded half is computed before the wait */
 constexpr int kTraceSlots = 48;         /* 0-3 reducer, 4 + 3r .. 6 + 3r rank r's producer, 28 done flags */
 
-/* Bounded wait that also gives up when another CTA has already recorded a failure. */
-template <bool GE>
-__device__ __forceinline__ bool chain_wait(const uint32_t *flag, uint32_t want, DevState *st, int *host_status,
-                                           unsigned long long timeout_ns)
-{
-    Deadline d;
-    for (;;) {
-        const uint32_t v = ld_acquire_u32(flag);
-        if (GE ? (v >= want) : (v == want)) return true;
-        if (d.expired(timeout_ns)) { fail(st, host_status, SIFAR_ERR_TIMEOUT); return false; }
-        if ((d.polls % 64u) == 0u && ld_relaxed_u32(&st->status) != 0u) return false;
-    }
-}
-
 template <int DT, int P, int MODE, bool TRACE>
 __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
 {
@@ -265,7 +251,7 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
                 if (threadIdx.x < 32) {
                     bool ok = true;
                     if (threadIdx.x < P)
-                        ok = chain_wait<false>(&cf->arrive[p][threadIdx.x], e, st, a.host_status, a.timeout_ns);
+                        ok = wait_flag_or_fail<false>(&cf->arrive[p][threadIdx.x], e, st, a.host_status, a.timeout_ns);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (threadIdx.x == 0) s_ok = ok;
                 }
@@ -361,9 +347,9 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
             if (threadIdx.x == 0) {
                 bool ok = true;
                 if (!no_ar && t > 1u) {
-                    ok = chain_wait<true>(&cf->ready, e - 1u, st, a.host_status, a.timeout_ns);
+                    ok = wait_flag_or_fail<true>(&cf->ready, e - 1u, st, a.host_status, a.timeout_ns);
                     if (ok && MODE == SIFAR_BARRIER_ONESHOT)
-                        ok = chain_wait<true>(&a.cs->done[rank], e - 1u, st, a.host_status, a.timeout_ns);
+                        ok = wait_flag_or_fail<true>(&a.cs->done[rank], e - 1u, st, a.host_status, a.timeout_ns);
                 }
                 SIFAR_TRACE(4 + 3 * rank);
                 if (ok) spin_ns(gen_delay_ns(a.w, rank, t));

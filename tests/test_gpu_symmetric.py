@@ -168,3 +168,30 @@ def test_context_is_usable_for_the_barrier_mode_after_a_persistent_chain(oracle,
         torch.cuda.synchronize()
         assert sf.sifar_status(ctx.h) == 0
         assert_bits_equal(out_to_numpy(out, n, BF16)[0], oracle.allreduce(xs, BF16), BF16, "after the chain")
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(oracle, mode):
+    """Ranks that are delayed by up to 1 ms against a 50 us limit: the waiting ranks give up, the kernel ends,
+    the status is sticky, and after a reset the context works again."""
+    P, n, steps = 4, 4096, 8
+    d = dict(synth.chain_workload("llama", P), delay_max_ns=1_000_000)
+    xs = synth.rank_inputs(P, n, BF16, seed=78, dist="uniform")
+    xs_dev = [to_device(x) for x in xs]
+    with Ctx(P, n, BF16, timeout_us=50) as ctx:
+        rings, _ = _rings(P, n, BF16, steps)
+        ch = sf.sifar_symchain_create(ctx.h, sf.make_workload(**d), n, mode, rings.data_ptr(), steps, steps)
+        sf.sifar_symchain_run(ch, 0)
+        torch.cuda.synchronize()
+        assert sf.sifar_status(ctx.h) == sf.ERR_TIMEOUT
+        assert sf.lib().sifar_get_stats  # the library still answers
+        assert sf._wl().sifar_symchain_run(ch, None) == sf.ERR_TIMEOUT      # refused: the status is sticky
+        sf.sifar_symchain_destroy(ch)
+        sf.sifar_reset(ctx.h, 0)
+        sf.sifar_set_timeout_us(ctx.h, 2_000_000)
+        assert sf.sifar_status(ctx.h) == 0
+        out = empty_out(n, BF16)
+        allreduce_via_pack(ctx, xs_dev, n, mode, out)
+        torch.cuda.synchronize()
+        assert sf.sifar_status(ctx.h) == 0
+        assert_bits_equal(out_to_numpy(out, n, BF16)[0], oracle.allreduce(xs, BF16), BF16, "after the reset")
