@@ -64,7 +64,8 @@ typedef enum {
    A timing floor; its results are not a sum. */
 enum { SIFAR_CHAIN_NO_ALLREDUCE = 3 };
 
-/* Bytes between two rows of an output ring for n elements (a multiple of 256, at least 16 bytes more than the row). */
+/* Bytes between two rows of an output ring for n elements (a multiple of 256, at least 512 bytes more than the
+   row: the persistent kernels work in whole warps of 16-byte units and write zeros behind the last element). */
 size_t sifar_chain_ring_stride(int dtype, size_t n);
 
 /*

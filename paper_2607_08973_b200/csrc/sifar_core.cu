@@ -792,8 +792,9 @@ extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
     if (const char *env = getenv("SIFAR_POLL_PACE_NS")) c->poll_pace_ns = (uint32_t)strtoul(env, nullptr, 10);
     cudaError_t e = cudaGetDevice(&c->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
-    c->plain_stride = round_up(max_elems * elem_size(dtype), 256);
-    c->slot_stride = round_up(slots_for(dtype, max_elems) * 16, 256);
+    /* kUnitPadBytes of slack: the persistent chain kernels work in whole warps of 16-byte units */
+    c->plain_stride = round_up(max_elems * elem_size(dtype) + kUnitPadBytes, 256);
+    c->slot_stride = round_up(slots_for(dtype, max_elems) * 16 + kUnitPadBytes, 256);
     const size_t plain_bytes = c->plain_stride * 2 * P, slot_bytes = c->slot_stride * 2 * P;
     if (e == cudaSuccess) e = cudaMalloc(&c->d_plain, plain_bytes);
     if (e == cudaSuccess) e = cudaMalloc(&c->d_slots, slot_bytes);

@@ -15,6 +15,7 @@
 namespace sifar {
 
 constexpr int kMaxRanks = SIFAR_MAX_RANKS;
+constexpr size_t kUnitPadBytes = 512;            /* 32 units of 16 bytes: room behind every rank buffer and ring row */
 constexpr uint32_t kEpochLimit = 0xFFFFFFFEu;    /* last usable call number                  */
 
 /*

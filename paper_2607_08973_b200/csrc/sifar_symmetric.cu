@@ -92,7 +92,9 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
     const uint32_t chunk = blockIdx.x / (uint32_t)P;
     SymFlags *cf = a.flags + chunk;
     const size_t n = (size_t)a.n;
-    const size_t nunits = (n + NE - 1) / NE;
+    /* whole warps of units (a partly filled warp was measured to slow its chunk down); units past the last
+       element carry zeros, and the rank buffers and result rows have room for them */
+    const size_t nunits = ((n + NE - 1) / NE + 31) / 32 * 32;
     const size_t n_io = nunits * NE;                                  /* result rows are padded to whole units */
     const size_t unit0 = (size_t)chunk * kSymThreads * a.K + threadIdx.x;
     char *my_ring = a.rings + (size_t)rank * a.ring_len * a.ring_stride;

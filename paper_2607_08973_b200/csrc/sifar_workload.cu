@@ -210,7 +210,10 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
     ChunkFlags *cf = a.chunks + chunk;
     const size_t n = (size_t)a.n;
     constexpr int EPU = (MODE == SIFAR_SPECULATIVE) ? ((DT == SIFAR_BF16) ? 6 : 3) : ((DT == SIFAR_BF16) ? 8 : 4);
-    const size_t nunits = (n + EPU - 1) / EPU;
+    /* Whole warps of units: a warp of which only some lanes have a unit was measured up to 0.4 us per step slower
+       (the ragged last chunk then set the pace of the whole result).  Units past the last element carry zeros;
+       the rank buffers and the ring rows have room for them. */
+    const size_t nunits = ((n + EPU - 1) / EPU + 31) / 32 * 32;
     const size_t n_io = nunits * EPU;         /* ring rows are padded: whole units are read and written */
     const size_t unit0 = (size_t)chunk * kChainThreads * a.K + threadIdx.x;
     __shared__ int s_ok;
@@ -523,9 +526,10 @@ static bool valid_workload(const sifar_workload *w)
 extern "C" size_t sifar_chain_ring_stride(int dtype, size_t n)
 {
     if (dtype != SIFAR_BF16 && dtype != SIFAR_F32) return 0;
-    /* room for one whole slot or vector past the last element: the persistent chain reads and writes its
-       ragged last unit in full (sub-sector stores and the loads that follow them are slow at the L2) */
-    return (n * elem_size(dtype) + 16 + 255) / 256 * 256;
+    /* room for a warp's worth of 16-byte units past the last element: the persistent chains read and write
+       whole units in whole warps (sub-sector stores, the loads that follow them, and partly filled warps were
+       all measured slow on the chain's critical path) */
+    return (n * elem_size(dtype) + kUnitPadBytes + 255) / 256 * 256;
 }
 
 template <int DT>
