@@ -308,7 +308,8 @@ def measure_symmetric(sf, torch, synth, ranks, n, name="llama", steps=ARS_PER_ST
     ranks, every mode and the floor without all-reduce; mis-speculation per rank for the speculative mode."""
     d = synth.chain_workload(name, ranks)
     res = {}
-    for mode in (sf.BARRIER_ONESHOT, sf.DUALBUF, sf.SPECULATIVE, sf.CHAIN_NO_ALLREDUCE):
+    names = {sf.SYMCHAIN_TWOSHOT: "twoshot", sf.CHAIN_NO_ALLREDUCE: "no_allreduce", **sf.MODE_NAMES}
+    for mode in (sf.BARRIER_ONESHOT, sf.SYMCHAIN_TWOSHOT, sf.DUALBUF, sf.SPECULATIVE, sf.CHAIN_NO_ALLREDUCE):
         ctx = sf.sifar_create(ranks, n, 0)
         stride = sf.sifar_chain_ring_stride(0, n)
         rings = torch.zeros(ranks * 2 * stride, dtype=torch.uint8, device="cuda")
@@ -326,7 +327,7 @@ def measure_symmetric(sf, torch, synth, ranks, n, name="llama", steps=ARS_PER_ST
             stt = sf.sifar_get_stats(ctx)
             r["misspeculated_steps_per_rank"] = [round(x / ((warm + runs) * steps), 3) for x in rt]
             r["slot_reloads_per_call"] = round(stt["slot_reloads"] / max(1, stt["calls"]), 1)
-        res[sf.MODE_NAMES.get(mode, "no_allreduce")] = r
+        res[names[mode]] = r
         sf.sifar_symchain_destroy(ch)
         sf.sifar_destroy(ctx)
     return res

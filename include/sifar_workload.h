@@ -64,6 +64,10 @@ typedef enum {
    A timing floor; its results are not a sum. */
 enum { SIFAR_CHAIN_NO_ALLREDUCE = 3 };
 
+/* Fifth "mode", sifar_symchain_create only: the twoshot baseline (reduce-scatter, barrier, all-gather;
+   Section 3.1), which needs the P readers of that chain to mean anything. */
+enum { SIFAR_SYMCHAIN_TWOSHOT = 4 };
+
 /* Bytes between two rows of an output ring for n elements (a multiple of 256, at least 512 bytes more than the
    row: the persistent kernels work in whole warps of 16-byte units and write zeros behind the last element). */
 size_t sifar_chain_ring_stride(int dtype, size_t n);
@@ -138,8 +142,9 @@ int sifar_chain_destroy(sifar_chain *chain);
  * one-reader chains, P times.
  *   out_rings      device, P x ring_len rows of sifar_chain_ring_stride() bytes, caller-owned;
  *                  rank r's copy of out^t lands in row r * ring_len + (t-1) mod ring_len
- *   other arguments as for sifar_chain_create (mode may be SIFAR_CHAIN_NO_ALLREDUCE: every rank's
- *   operation feeds on its own partial, the timing floor)
+ *   other arguments as for sifar_chain_create (mode may also be SIFAR_CHAIN_NO_ALLREDUCE: every rank's
+ *   operation feeds on its own partial, the timing floor; or SIFAR_SYMCHAIN_TWOSHOT: every rank reduces
+ *   1/P of each chunk for all, a second barrier, then every rank reads the reduced chunk)
  * The chain owns the context exclusively until it is destroyed.
  */
 typedef struct sifar_symchain sifar_symchain;   /* opaque */

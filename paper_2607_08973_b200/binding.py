@@ -165,6 +165,7 @@ def sifar_noalloc_max_elems() -> int:
 # ---------------------------------------------------------------------------
 CHAIN_STREAMS, CHAIN_GRAPH, CHAIN_PERSISTENT = 0, 1, 2
 CHAIN_NO_ALLREDUCE = 3
+SYMCHAIN_TWOSHOT = 4
 IMPL_NAMES = {CHAIN_STREAMS: "streams", CHAIN_GRAPH: "graph", CHAIN_PERSISTENT: "persistent"}
 
 

@@ -18,6 +18,10 @@
  *   DUALBUF         : store into parity buffer, arrival flag; wait for P flags; load, sum
  *   SPECULATIVE     : store tagged slots; load all P copies at once, accept a slot iff
  *                     its tag is this call's number, re-load the stale ones
+ *   TWOSHOT         : the paper's other baseline (Section 3.1): store, arrival flag; wait for P flags;
+ *                     reduce 1/P of the chunk for everybody (reduce-scatter); second barrier; read the
+ *                     whole reduced chunk (all-gather).  The second barrier also covers the reuse of the
+ *                     single buffer: a rank passes it only after every rank's reads of the partials.
  * so ranks drift against each other as real GPUs do, and a rank mis-speculates
  * exactly when a peer is behind it.  A thread keeps the same units in every step;
  * the speculative mode needs no CTA-wide barrier at all: the write-after-read
@@ -40,6 +44,7 @@ namespace sifar {
 
 constexpr int kSymThreads = 128;
 constexpr int kSymNoAllreduce = SIFAR_CHAIN_NO_ALLREDUCE;
+constexpr int kSymTwoshot = SIFAR_SYMCHAIN_TWOSHOT;
 
 /* Flags of one chunk: what the P CTAs that own it tell each other. */
 struct __align__(128) SymFlags {
@@ -86,6 +91,8 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
     DevState *st = a.st;
     constexpr bool no_ar = (MODE == kSymNoAllreduce);
     constexpr bool spec = (MODE == SIFAR_SPECULATIVE);
+    constexpr bool two = (MODE == kSymTwoshot);
+    constexpr bool single = (MODE == SIFAR_BARRIER_ONESHOT || two);      /* one buffer per rank instead of two */
     constexpr int NW = spec ? 3 : 4;                                  /* words per unit */
     constexpr int NE = NW * ((DT == SIFAR_BF16) ? 2 : 1);             /* elements per unit */
     const uint32_t rank = blockIdx.x % (uint32_t)P;                   /* the P CTAs of a chunk are neighbours (one cluster) */
@@ -118,8 +125,7 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
         const char *prev_mem = no_ar ? a.plain + ((size_t)(p ^ 1u) * P + rank) * a.plain_stride
                                      : my_ring + (size_t)((t + a.ring_len - 2u) % a.ring_len) * a.ring_stride;
         uint4 *dst = spec ? reinterpret_cast<uint4 *>(a.slots + ((size_t)p * P + rank) * a.slot_stride)
-                          : reinterpret_cast<uint4 *>(a.plain + ((size_t)(MODE == SIFAR_BARRIER_ONESHOT ? 0u : p) * P + rank)
-                                                                    * a.plain_stride);
+                          : reinterpret_cast<uint4 *>(a.plain + ((size_t)(single ? 0u : p) * P + rank) * a.plain_stride);
 
         /* ---- 1. the rank's next operation: the seeded half first, it needs nothing from anybody ---- */
         float z0[NE];
@@ -168,8 +174,7 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
 #pragma unroll
         for (int r = 0; r < P; ++r)
             src[r] = spec ? reinterpret_cast<const uint4 *>(a.slots + ((size_t)p * P + r) * a.slot_stride)
-                          : reinterpret_cast<const uint4 *>(a.plain + ((size_t)(MODE == SIFAR_BARRIER_ONESHOT ? 0u : p) * P + r)
-                                                                          * a.plain_stride);
+                          : reinterpret_cast<const uint4 *>(a.plain + ((size_t)(single ? 0u : p) * P + r) * a.plain_stride);
         if (!spec) {
             /* arrival flag of this rank (release), then the top barrier: all P ranks' flags (acquire) */
             __syncthreads();
@@ -184,6 +189,41 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
             __syncthreads();
             if (!s_ok) { alive = false; break; }
         }
+        if constexpr (two) {
+            /* ---- 3a. reduce-scatter: this rank reduces its share of the chunk's units for everybody ---- */
+            uint4 *red = reinterpret_cast<uint4 *>(a.plain + (size_t)P * a.plain_stride);   /* parity 1, rank 0: unused here */
+            const bool mine = (threadIdx.x * (uint32_t)P / kSymThreads == rank);
+            for (uint32_t k = 0; k < a.K; ++k) {
+                const size_t u = unit0 + (size_t)k * kSymThreads;
+                if (u >= nunits) break;
+                if (mine) {
+                    uint4 x[P];
+#pragma unroll
+                    for (int r = 0; r < P; ++r) x[r] = ld_slot(src[r] + u);
+                    st_slot(red + u, sum_vec<DT, P>(x, true));
+                }
+            }
+            /* second barrier: all P shares of the chunk are reduced (the done flags serve as its arrival flags) */
+            __syncthreads();
+            if (threadIdx.x == 0) st_release_u32(&cf->done[rank], e);
+            if (threadIdx.x < 32) {
+                bool ok = true;
+                if (threadIdx.x < P)
+                    ok = wait_flag_or_fail<false>(&cf->done[threadIdx.x], e, st, a.host_status, a.timeout_ns);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (threadIdx.x == 0) s_ok = ok;
+            }
+            __syncthreads();
+            if (!s_ok) { alive = false; break; }
+            /* ---- 3b. all-gather: every rank takes the whole reduced chunk ---- */
+            for (uint32_t k = 0; k < a.K; ++k) {
+                const size_t u = unit0 + (size_t)k * kSymThreads;
+                if (u >= nunits) break;
+                const uint4 o = ld_slot(red + u);
+                store_vec_result<DT>(row, u, n_io, o);
+                if (k == 0) { prevw[0] = o.x; prevw[1] = o.y; prevw[2] = o.z; prevw[NW - 1] = o.w; }
+            }
+        } else {
         /* ---- 3. pull all P partials and reduce in rank order ---- */
         bool retried = false;
         for (uint32_t k = 0; k < a.K; ++k) {
@@ -220,6 +260,7 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
             __syncthreads();
             if (threadIdx.x == 0) st_release_u32(&cf->done[rank], e);
         }
+        }   /* !two */
         if (threadIdx.x == 0) my_stamps[s + 1u] = globaltimer_ns();
         }   /* !no_ar */
     }
@@ -267,6 +308,7 @@ static const void *sym_kernel_p(int mode)
     case SIFAR_BARRIER_ONESHOT: return (const void *)k_sym<DT, P, SIFAR_BARRIER_ONESHOT>;
     case SIFAR_DUALBUF:         return (const void *)k_sym<DT, P, SIFAR_DUALBUF>;
     case SIFAR_SPECULATIVE:     return (const void *)k_sym<DT, P, SIFAR_SPECULATIVE>;
+    case kSymTwoshot:           return (const void *)k_sym<DT, P, kSymTwoshot>;
     default:                    return (const void *)k_sym<DT, P, kSymNoAllreduce>;
     }
 }
@@ -385,7 +427,7 @@ extern "C" sifar_symchain *sifar_symchain_create(sifar_ctx *c, const sifar_workl
                                                  void *out_rings, int ring_len, int steps_per_run)
 {
     if (!c || !w || w->kind < 0 || w->kind > 2 || w->delay_max_ns > 1000000u || n == 0 || n > c->max_elems ||
-        mode < 0 || mode > kSymNoAllreduce || !out_rings || ((uintptr_t)out_rings & 15u) || ring_len < 2 ||
+        mode < 0 || mode > kSymTwoshot || !out_rings || ((uintptr_t)out_rings & 15u) || ring_len < 2 ||
         steps_per_run < 2 || (steps_per_run & 1) || steps_per_run % ring_len != 0) {
         set_error("sifar_symchain_create: bad argument (need 1 <= n <= max_elems, ring_len >= 2 dividing an even "
                   "steps_per_run, delay_max_ns <= 1000000)");
