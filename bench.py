@@ -262,6 +262,35 @@ def measure_roofline(sf, torch, P_, n, mode, warmup, iters, dtype=0, nctx=6):
     return float(np.mean(times)), float(np.median(times)), len(times) * nctx
 
 
+def measure_pack(sf, torch, P_, n, mode, reps=8):
+    """Producer-side store path: all P ranks pack at the same time, one stream per rank; device time from the
+    common start to the last rank's end, and the bytes read and written."""
+    srcs = [torch.randn(n, device="cuda").to(torch.bfloat16) for _ in range(P_)]
+    ctx = sf.sifar_create(P_, n, 0)
+    streams = [torch.cuda.Stream() for _ in range(P_)]
+    main = torch.cuda.Stream()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ts = []
+    for _ in range(reps):
+        sf.sifar_spin(200_000, main.cuda_stream)            # lets the host enqueue all P launches ahead
+        ev0.record(main)
+        joins = []
+        for r in range(P_):
+            streams[r].wait_event(ev0)
+            sf.sifar_pack(ctx, r, srcs[r].data_ptr(), n, mode, streams[r].cuda_stream)
+            j = torch.cuda.Event()
+            j.record(streams[r])
+            joins.append(j)
+        for j in joins:
+            main.wait_event(j)
+        ev1.record(main)
+        main.synchronize()
+        ts.append(ev0.elapsed_time(ev1) * 1e-3)
+    sf.sifar_destroy(ctx)
+    per_rank = n * 2 + (sf.sifar_slot_count(0, n) * 16 if mode == sf.SPECULATIVE else n * 2)
+    return float(np.median(ts[2:])), P_ * per_rank
+
+
 def measure_e2e(sf, torch, synth, n, mode, warmup, steps):
     """Host buffers in, host buffer out, through sifar_allreduce_host: one decode step = 64 calls."""
     ctx = sf.sifar_create(P, n, 0)
@@ -441,6 +470,10 @@ def run_gpu(args) -> None:
         ab = sf.sifar_algorithmic_bytes(P, sf.BF16, 4 * LARGE_N, sf.SPECULATIVE)
         roof["at_64MiB_per_rank"] = {"kernel_us": round(ms_ * 1e6, 2), "achieved": round(ab / ms_ / 1e9, 1),
                                      "frac": round(ab / ms_ / 1e9 / peak_gbs, 4)}
+        pk_s, pk_bytes = measure_pack(sf, torch, P, LARGE_N, sf.SPECULATIVE)
+        roof["producer_store"] = {"kernel": "k_pack<bf16,speculative> x 8 ranks on 8 streams", "us": round(pk_s * 1e6, 1),
+                                  "bytes": pk_bytes, "achieved": round(pk_bytes / pk_s / 1e9, 1),
+                                  "frac": round(pk_bytes / pk_s / 1e9 / peak_gbs, 4)}
         roof["traffic"] = NCU_TRAFFIC_BYTES
         roof["traffic_source"] = "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel and size"
         alg_d = sf.sifar_algorithmic_bytes(P, sf.BF16, n, sf.SPECULATIVE) * ARS_PER_STEP
