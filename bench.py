@@ -196,9 +196,9 @@ class Chain:
         self.sf.sifar_destroy(self.ctx)
 
 
-def measure_modes(sf, torch, synth, n, warmup, reps, impls, modes, rounds=3):
+def measure_modes(sf, torch, synth, n, warmup, reps, impls, modes, rounds=3, name="llama", steps=ARS_PER_STEP):
     """Interleaved A/B/C measurement: every (impl, mode) chain is visited `rounds` times."""
-    chains = {(i, m): Chain(sf, torch, synth, n, m, i) for i in impls for m in modes}
+    chains = {(i, m): Chain(sf, torch, synth, n, m, i, steps=steps, name=name) for i in impls for m in modes}
     for c in chains.values():
         for _ in range(warmup):
             c.run()
@@ -213,7 +213,7 @@ def measure_modes(sf, torch, synth, n, warmup, reps, impls, modes, rounds=3):
     for (i, m), c in chains.items():
         name = f"{sf.IMPL_NAMES[i]}/{sf.MODE_NAMES.get(m, 'no_allreduce')}"
         step_us = float(np.median(acc[(i, m)]["step_us"]))
-        r = {"decode_step_us": round(step_us, 2), "us_per_allreduce_mean": round(step_us / ARS_PER_STEP, 3)}
+        r = {"decode_step_us": round(step_us, 2), "us_per_allreduce_mean": round(step_us / steps, 3)}
         if acc[(i, m)]["iv"]:
             iv = np.concatenate(acc[(i, m)]["iv"])
             r.update(p50_us=round(pct(iv, 50), 3), p99_us=round(pct(iv, 99), 3))
@@ -447,6 +447,11 @@ def run_gpu(args) -> None:
                 str(b): measure_modes(sf, torch, synth, HIDDEN * b, args.warmup, max(8, args.steps // 8),
                                       (sf.CHAIN_PERSISTENT, sf.CHAIN_GRAPH), modes)
                 for b in (2, 4, 8, 16)}
+            # config 3: MoE-shaped step, 120 dependent all-reduces, 1 % outliers
+            detail["moe_by_batch_tokens"] = {
+                str(b): measure_modes(sf, torch, synth, HIDDEN * b, 3, 6, (sf.CHAIN_PERSISTENT, sf.CHAIN_GRAPH), modes,
+                                      rounds=2, name="moe", steps=120)
+                for b in (1, 8, 32, 64)}
             detail["streams"] = measure_modes(sf, torch, synth, n, 3, 8, (sf.CHAIN_STREAMS,), modes, rounds=2)
             detail["payload_sweep"] = payload_sweep(sf, torch)
             detail["retry_overhead"] = retry_overhead(sf, torch, synth)
