@@ -43,3 +43,42 @@ def test_random_shapes_and_bit_patterns(oracle, P, n, dtype, mode, seed, calls):
                     assert np.array_equal(got[~nan], want[~nan]) and np.all(got[nan] == 0x7FFF)
                 else:
                     assert_bits_equal(got, want, dtype, f"P={P} n={n} mode={mode}")
+
+
+@settings(max_examples=40, deadline=None, suppress_health_check=list(HealthCheck))
+@given(P=st.integers(1, 8), n=st.integers(1, 3000), dtype=st.sampled_from([BF16, F32]), mode=st.integers(0, 4),
+       kind=st.integers(0, 2), seed=st.integers(0, 2 ** 31 - 1), one_reader=st.booleans(),
+       delay=st.sampled_from([0, 0, 3000]))
+def test_random_decode_chains(oracle, P, n, dtype, mode, kind, seed, one_reader, delay):
+    """Random workloads through the persistent chains (one reader, P readers, twoshot): every step of two runs."""
+    if mode == 3 or (one_reader and mode == 4):
+        mode = sf.SPECULATIVE                 # 3 is the floor without all-reduce, 4 exists with P readers only
+    d = dict(kind=kind, seed=seed, scale=1.0 / P if kind != 1 else 1.0, sigma=0.25, outlier_mod=(0, 7)[seed & 1],
+             delay_max_ns=delay)
+    steps = 4
+    want = oracle.chain(oracle.Workload(d["kind"], d["seed"], d["scale"], d["sigma"], d["outlier_mod"],
+                                        d["delay_max_ns"]), P, n, dtype, 2 * steps)
+    stride = sf.sifar_chain_ring_stride(dtype, n)
+    nd = np.uint16 if dtype == BF16 else np.float32
+    copies = 1 if one_reader else P
+    with Ctx(P, n, dtype, timeout_us=5_000_000) as ctx:
+        rings = torch.zeros(copies * steps * stride, dtype=torch.uint8, device="cuda")
+        w = sf.make_workload(**d)
+        if one_reader:
+            ch = sf.sifar_chain_create(ctx.h, w, n, mode, sf.CHAIN_PERSISTENT, rings.data_ptr(), steps, steps)
+            run, destroy = sf.sifar_chain_run, sf.sifar_chain_destroy
+        else:
+            ch = sf.sifar_symchain_create(ctx.h, w, n, mode, rings.data_ptr(), steps, steps)
+            run, destroy = sf.sifar_symchain_run, sf.sifar_symchain_destroy
+        try:
+            for k in range(2):
+                run(ch, 0)
+                torch.cuda.synchronize()
+                assert sf.sifar_status(ctx.h) == 0
+                h = rings.cpu().numpy().reshape(copies, steps, stride)[:, :, : n * nd().itemsize].copy().view(nd)
+                for r in range(copies):
+                    for s in range(steps):
+                        assert_bits_equal(h[r, s], want[k * steps + s], dtype,
+                                          f"P={P} n={n} mode={mode} kind={kind} copy {r} step {k * steps + s + 1}")
+        finally:
+            destroy(ch)
