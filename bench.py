@@ -40,8 +40,8 @@ sys.path.insert(0, ROOT)
 METRIC = "p50 us per P=8 emulated all-reduce (decode payload), with HBM roofline fraction at a 16 MiB payload"
 P, HIDDEN, ARS_PER_STEP = 8, 4096, 64
 LARGE_N = 8 << 20                      # 16 MiB of bf16 per rank
-# DRAM bytes per launch of k_reduce_spec<bf16,8> at LARGE_N from one ncu capture: 179.01 MB read + 11.40 MB written
-NCU_TRAFFIC_BYTES = 190_412_544
+# DRAM bytes per launch of k_reduce_spec<bf16,8> at LARGE_N from one ncu capture: 179.00 MB read + 12.66 MB written
+NCU_TRAFFIC_BYTES = 191_657_728
 
 
 def read_peaks() -> tuple[float, str]:
