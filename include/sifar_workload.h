@@ -111,7 +111,7 @@ int sifar_chain_chunks(sifar_chain *chain);
  * unless stated) written by the CTAs that own chunk 0:
  *   reducer, thread 0:  [0] enters the step      [1] arrival flags seen (speculative: its warp's slots valid)
  *                       [2] whole chunk reduced  [3] ready flag released
- *                       [28] done flags released (BARRIER_ONESHOT, last reducer CTA only)
+ *                       [28] done flags released (BARRIER_ONESHOT)
  *                       [29] number of slot re-loads of thread 0 in this step (a count)
  *                       [30..37] end of its first eight re-poll rounds (speculative)
  *   reducer, lane 0 of warp w:   [38+w] the warp's slots validated (speculative)

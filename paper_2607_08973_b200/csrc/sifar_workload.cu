@@ -10,7 +10,7 @@
  * what differs between the modes is exactly the synchronization they perform:
  *
  *   BARRIER_ONESHOT : ready -> [done wait] produce -> arrival flag -> flag poll
- *                     -> load/sum/store -> ready; all reducer CTAs arrive, done flags
+ *                     -> load/sum/store -> ready, the chunk's P done flags
  *   DUALBUF         : ready -> produce -> arrival flag -> flag poll -> load/sum/store -> ready
  *   SPECULATIVE     : ready -> produce tagged slots -> load/validate/sum/store -> ready
  *
@@ -139,14 +139,12 @@ struct __align__(128) ChunkFlags {
     uint32_t ready;                 /* call number whose result chunk is published                  */
     uint32_t pad0[7];
     uint32_t arrive[2][8];          /* per parity, per rank: this chunk of the rank's partial stored */
-    uint32_t pad1[8];
+    uint32_t done[8];               /* per rank: the chunk's reducer has finished reading call e (bottom barrier) */
 };
 
 struct __align__(128) ChainDev {
-    uint32_t bottom_count;          /* reducer CTAs that finished reading (monotonic)               */
     uint32_t exit_count;            /* CTAs that left the kernel (monotonic)                        */
-    uint32_t pad0[30];
-    uint32_t done[32];              /* bottom barrier, per rank                                     */
+    uint32_t pad0[31];
 };
 
 struct PersistArgs {
@@ -167,7 +165,7 @@ struct PersistArgs {
     uint32_t steps;
     uint32_t C;                     /* chunks = reducer CTAs               */
     uint32_t K;                     /* units per thread and step           */
-    uint32_t bottom_base, exit_base;
+    uint32_t exit_base;
     uint32_t clustered;             /* role layout, see k_chain */
     PollShape poll;
     ChainDev *cs;
@@ -314,13 +312,12 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
                     st_relaxed_u32(&a.retry_steps[s], 1u);
                 }
                 if (stamper) my_stamps[s + 1u] = globaltimer_ns();
-                if (MODE == SIFAR_BARRIER_ONESHOT) {
-                    /* bottom barrier, reducer side: last CTA to finish reading releases the done flags */
-                    const uint32_t arrived = atom_add_acq_rel_u32(&a.cs->bottom_count, 1u) + 1u;
-                    if (arrived == a.bottom_base + (s + 1u) * C)
-                        for (int r = 0; r < P; ++r) st_release_u32(&a.cs->done[r], e);
-                    SIFAR_TRACE(28);
-                }
+            }
+            if (MODE == SIFAR_BARRIER_ONESHOT) {
+                /* bottom barrier, reducer side, block by block as the top barrier: the chunk has been read, its
+                   P done flags are released (one lane each; every thread has passed the barrier above) */
+                if (threadIdx.x < P) st_release_u32(&cf->done[threadIdx.x], e);
+                SIFAR_TRACE(28);
             }
         } else {
             /* ---------------- rank `rank`, chunk `chunk` of the next operation ---------------- */
@@ -352,7 +349,7 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
                 if (!no_ar && t > 1u) {
                     ok = wait_flag_or_fail<true>(&cf->ready, e - 1u, st, a.host_status, a.timeout_ns);
                     if (ok && MODE == SIFAR_BARRIER_ONESHOT)
-                        ok = wait_flag_or_fail<true>(&a.cs->done[rank], e - 1u, st, a.host_status, a.timeout_ns);
+                        ok = wait_flag_or_fail<true>(&cf->done[rank], e - 1u, st, a.host_status, a.timeout_ns);
                 }
                 SIFAR_TRACE(4 + 3 * rank);
                 if (ok) spin_ns(gen_delay_ns(a.w, rank, t));
@@ -820,7 +817,6 @@ extern "C" int sifar_chain_run(sifar_chain *ch, void *stream)
         a.base_epoch = ch->base_epoch; a.steps = (uint32_t)ch->steps;
         a.C = ch->C; a.K = ch->K;
         a.poll = poll_shape_for(c, ch->n);
-        a.bottom_base = ch->runs * (uint32_t)ch->steps * ch->C;
         a.exit_base = ch->runs * (uint32_t)ch->grid;
         a.cs = ch->d_cs; a.chunks = ch->d_chunks; a.stamps = ch->d_stamps; a.retry_steps = ch->d_retry_steps;
         a.trace = ch->trace_on ? ch->d_trace : nullptr;
