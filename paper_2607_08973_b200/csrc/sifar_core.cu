@@ -100,8 +100,11 @@ __device__ __forceinline__ void publish_call(DevState *st, uint32_t e, int P)
     atomicAdd(&st->stats[kStatCalls], 1ull);                          /* result unused: fire and forget */
     if (MODE == SIFAR_SPECULATIVE && ld_relaxed_u32(&st->retry_epoch) == e)
         atomicAdd(&st->stats[kStatCallsWithRetry], 1ull);
-    if (MODE == SIFAR_BARRIER_ONESHOT)
-        for (int r = 0; r < P; ++r) st_release_u32(&st->done[r], e);
+    if (MODE == SIFAR_BARRIER_ONESHOT) {
+        /* one fence, then the P done flags: P release stores in a row would each wait for the one before */
+        __threadfence();
+        for (int r = 0; r < P; ++r) st_relaxed_u32(&st->done[r], e);
+    }
     /* readers of the call number are ordered after this kernel by the stream or by an event */
     st_relaxed_u32(&st->epoch, e);
 }
@@ -616,8 +619,10 @@ __global__ void k_empty_call(DevState *st, int mode, int P)
     if (es.y != 0u) return;
     const uint32_t e = es.x + 1u;
     st->stats[kStatCalls] += 1ull;
-    if (mode == SIFAR_BARRIER_ONESHOT)
-        for (int r = 0; r < P; ++r) st_release_u32(&st->done[r], e);
+    if (mode == SIFAR_BARRIER_ONESHOT) {
+        __threadfence();
+        for (int r = 0; r < P; ++r) st_relaxed_u32(&st->done[r], e);
+    }
     st_release_u32(&st->epoch, e);
 }
 
