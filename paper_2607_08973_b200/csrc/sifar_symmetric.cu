@@ -80,7 +80,7 @@ struct SymArgs {
     PollShape poll;
     SymDev *cs;
     SymFlags *flags;                /* C */
-    unsigned long long *stamps;     /* [rank][chunk][steps + 1] */
+    unsigned long long *stamps;     /* [rank][chunk][warp][steps + 1] */
     uint32_t *retry_marks;          /* [rank][steps]: 1 if the rank re-loaded a slot in that step */
     unsigned long long *rank_retries; /* [P] cumulative (rank, step) pairs with a re-load */
 };
@@ -105,14 +105,18 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
     const size_t n_io = nunits * NE;                                  /* result rows are padded to whole units */
     const size_t unit0 = (size_t)chunk * kSymThreads * a.K + threadIdx.x;
     char *my_ring = a.rings + (size_t)rank * a.ring_len * a.ring_stride;
-    unsigned long long *my_stamps = a.stamps + ((size_t)rank * a.C + chunk) * (a.steps + 1u);
+    /* Stamps per warp: without a CTA-wide barrier (speculative mode has none) the warps of a CTA are pipelines
+       of their own, and a chunk of a result is complete when the last of them is; the host takes the maximum. */
+    constexpr uint32_t kWarps = kSymThreads / 32;
+    const bool stamper = (threadIdx.x & 31u) == 0u;
+    unsigned long long *my_stamps = a.stamps + (((size_t)rank * a.C + chunk) * kWarps + (threadIdx.x >> 5)) * (a.steps + 1u);
     __shared__ int s_ok;
     unsigned reloads = 0;
     bool alive = true;
     uint32_t prevw[NW];                                               /* this thread's first unit of the previous result */
 #pragma unroll
     for (int j = 0; j < NW; ++j) prevw[j] = 0u;
-    if (threadIdx.x == 0) my_stamps[0] = globaltimer_ns();
+    if (stamper) my_stamps[0] = globaltimer_ns();
 
     for (uint32_t s = 0; s < a.steps && alive; ++s) {
         const uint32_t e = a.e0 + 1u + s;
@@ -168,7 +172,7 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
         }
         if constexpr (no_ar) {
             __syncthreads();
-            if (threadIdx.x == 0) my_stamps[s + 1u] = globaltimer_ns();
+            if (stamper) my_stamps[s + 1u] = globaltimer_ns();
         } else {
         const uint4 *src[P];
 #pragma unroll
@@ -261,7 +265,7 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
             if (threadIdx.x == 0) st_release_u32(&cf->done[rank], e);
         }
         }   /* !two */
-        if (threadIdx.x == 0) my_stamps[s + 1u] = globaltimer_ns();
+        if (stamper) my_stamps[s + 1u] = globaltimer_ns();
         }   /* !no_ar */
     }
 
@@ -409,7 +413,7 @@ static int sym_setup(sifar_symchain *ch)
         if (err == cudaSuccess && (size_t)max_clusters >= C) ch->clustered = true;
         else cudaGetLastError();
     }
-    const size_t nstamps = (size_t)P * C * (ch->steps + 1);
+    const size_t nstamps = (size_t)P * C * (kSymThreads / 32) * (ch->steps + 1);
     SIFAR_CUDA(cudaMalloc(&ch->d_cs, sizeof(SymDev)));
     SIFAR_CUDA(cudaMalloc(&ch->d_flags, sizeof(SymFlags) * C));
     SIFAR_CUDA(cudaMalloc(&ch->d_stamps, sizeof(unsigned long long) * nstamps));
@@ -515,14 +519,15 @@ static int sym_stamps(sifar_symchain *ch, int r0, int r1, unsigned long long *st
 {
     SIFAR_CUDA(cudaDeviceSynchronize());
     const size_t per = (size_t)ch->steps + 1;
-    std::vector<unsigned long long> all(per * ch->C * ch->ctx->P);
+    const size_t pipes = (size_t)ch->C * (kSymThreads / 32);         /* chunks x warps of one rank */
+    std::vector<unsigned long long> all(per * pipes * ch->ctx->P);
     SIFAR_CUDA(cudaMemcpy(all.data(), ch->d_stamps, sizeof(unsigned long long) * all.size(), cudaMemcpyDeviceToHost));
     for (size_t s = 0; s < per; ++s) {
         unsigned long long v = 0;
         bool have = false;
         for (int r = r0; r < r1; ++r)
-            for (uint32_t c = 0; c < ch->C; ++c) {
-                const unsigned long long x = all[((size_t)r * ch->C + c) * per + s];
+            for (size_t c = 0; c < pipes; ++c) {
+                const unsigned long long x = all[((size_t)r * pipes + c) * per + s];
                 if (!have) { v = x; have = true; }
                 else v = (s == 0) ? (x < v ? x : v) : (x > v ? x : v);
             }
