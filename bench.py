@@ -328,6 +328,10 @@ def payload_sweep(sf, torch, exps=range(10, 26), ranks=(2, 4, 8)):
                     mean_s, med_s, _ = measure_roofline(sf, torch, P_, n, mode, 2, 5, dtype=dtype, nctx=nctx)
                     alg = sf.sifar_algorithmic_bytes(P_, dtype, n, mode)
                     row[sf.MODE_NAMES[mode]] = {"us": round(med_s * 1e6, 2), "GBps": round(alg / med_s / 1e9, 1)}
+                # the size-adaptive choice between the two barrier-free modes, and what it costs against the better one
+                pick = sf.MODE_NAMES[sf.sifar_mode_for_payload(P_, dtype, n)]
+                best = min(row["dualbuf"]["us"], row["speculative"]["us"])
+                row["adaptive"] = {"mode": pick, "us": row[pick]["us"], "over_best_pct": round(100 * (row[pick]["us"] / best - 1), 1)}
                 rows.append(row)
     return rows
 

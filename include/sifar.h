@@ -193,6 +193,18 @@ int sifar_reset(sifar_ctx *ctx, void *stream);
 int sifar_debug_set_epoch(sifar_ctx *ctx, unsigned calls_so_far);
 
 /*
+ * Size-adaptive choice between the two barrier-free modes.  The paper has no
+ * counterpart: it targets decode payloads of 8-32 KB (Section 5), where the tags
+ * of the speculative slots cost nothing that matters.  For large payloads the
+ * tagged slots move a third more bytes than plain data, which is what bounds the
+ * reducer there.  Returns SIFAR_SPECULATIVE while all P partials together stay
+ * below 16 MiB (the crossover measured on B200 for P = 2, 4 and 8, bf16 and fp32:
+ * 2 MiB per rank at P = 8, 8 MiB per rank at P = 2) and SIFAR_DUALBUF from there
+ * on; SIFAR_ERR_INVALID for a bad P or dtype.  Pure function, no device access.
+ */
+int sifar_mode_for_payload(int P, int dtype, size_t n);
+
+/*
  * Measurement hook for the retry-latency experiment (Section 7, "Retry Overhead":
  * latency of the no-retry case and what each further retry adds, obtained by
  * forcing a fixed number of retries).  With rounds = k > 0 the speculative reducer

@@ -50,6 +50,7 @@ def lib() -> ctypes.CDLL:
             "sifar_reset": (ci, [vp, vp]),
             "sifar_debug_set_epoch": (ci, [vp, cu]),
             "sifar_debug_force_retries": (ci, [vp, cu]),
+            "sifar_mode_for_payload": (ci, [ci, ci, sz]),
             "sifar_slot_count": (sz, [ci, sz]),
             "sifar_algorithmic_bytes": (sz, [ci, ci, sz, ci]),
             "sifar_last_error": (ctypes.c_char_p, []),
@@ -137,6 +138,13 @@ def sifar_reset(ctx: int, stream: int = 0) -> int:
 
 def sifar_debug_set_epoch(ctx: int, calls_so_far: int) -> int:
     return _check(lib().sifar_debug_set_epoch(ctx, calls_so_far))
+
+
+def sifar_mode_for_payload(P: int, dtype: int, n: int) -> int:
+    mode = lib().sifar_mode_for_payload(P, dtype, n)
+    if mode < 0:
+        raise SifarError(mode, sifar_last_error())
+    return mode
 
 
 def sifar_debug_force_retries(ctx: int, rounds: int) -> int:

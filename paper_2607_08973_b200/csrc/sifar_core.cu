@@ -793,6 +793,16 @@ extern "C" size_t sifar_algorithmic_bytes(int P, int dtype, size_t n, int mode)
     return (size_t)P * per_rank + payload + flags;
 }
 
+extern "C" int sifar_mode_for_payload(int P, int dtype, size_t n)
+{
+    if (P < 1 || P > kMaxRanks || !valid_dtype(dtype)) {
+        set_error("sifar_mode_for_payload: need 1 <= P <= %d and a known dtype", kMaxRanks);
+        return SIFAR_ERR_INVALID;
+    }
+    constexpr size_t kSpeculativeBelowBytes = (size_t)16 << 20;     /* all P partials together */
+    return (size_t)P * n * elem_size(dtype) < kSpeculativeBelowBytes ? SIFAR_SPECULATIVE : SIFAR_DUALBUF;
+}
+
 extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
 {
     g_error[0] = 0;

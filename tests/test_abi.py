@@ -35,6 +35,23 @@ def test_geometry_helpers_need_no_gpu():
     assert sf.sifar_algorithmic_bytes(8, sf.BF16, 4096, sf.BARRIER_ONESHOT) == 9 * 8192 + 64
 
 
+def test_size_adaptive_mode_choice_needs_no_gpu():
+    import pytest
+    from paper_2607_08973_b200 import binding as sf
+    # speculative while all P partials together stay below 16 MiB, dual-buffered from there on
+    assert sf.sifar_mode_for_payload(8, sf.BF16, 4096) == sf.SPECULATIVE
+    assert sf.sifar_mode_for_payload(8, sf.BF16, (1 << 20) - 1) == sf.SPECULATIVE
+    assert sf.sifar_mode_for_payload(8, sf.BF16, 1 << 20) == sf.DUALBUF            # 8 x 2 MiB
+    assert sf.sifar_mode_for_payload(2, sf.BF16, (1 << 22) - 1) == sf.SPECULATIVE
+    assert sf.sifar_mode_for_payload(2, sf.BF16, 1 << 22) == sf.DUALBUF            # 2 x 8 MiB
+    assert sf.sifar_mode_for_payload(8, sf.F32, (1 << 19) - 1) == sf.SPECULATIVE
+    assert sf.sifar_mode_for_payload(8, sf.F32, 1 << 19) == sf.DUALBUF
+    assert sf.sifar_mode_for_payload(1, sf.BF16, 0) == sf.SPECULATIVE
+    for bad in ((0, sf.BF16, 1), (9, sf.BF16, 1), (2, 7, 1)):
+        with pytest.raises(sf.SifarError):
+            sf.sifar_mode_for_payload(*bad)
+
+
 def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     from paper_2607_08973_b200 import binding as sf
     monkeypatch.setattr(sf, "_lib", None)
