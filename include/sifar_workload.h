@@ -30,6 +30,14 @@
  *       x_r^t[i]   = ((int(out^{t-1}[i]) + k) mod 129, taken in [0,128]) - 64
  * delay_max_ns > 0: before storing, rank r at step t busy-waits a seeded time
  * uniform on [0, delay_max_ns] (skewed arrival); values are unaffected.
+ *
+ * Two families of chains run these steps:
+ *   sifar_chain_*     one reader: P producers feed one all-reduce whose single result
+ *                     feeds all P producers again (streams, CUDA graph, or one
+ *                     persistent kernel), which is what sifar_allreduce computes;
+ *   sifar_symchain_*  P readers: every rank runs its operation and its own
+ *                     pull-and-reduce and keeps its own copy of the result, as every
+ *                     GPU of the paper's system does; also carries the twoshot baseline.
  */
 #ifndef SIFAR_WORKLOAD_H
 #define SIFAR_WORKLOAD_H
