@@ -26,7 +26,8 @@
  * P*x, integer inputs against exact integer arithmetic in every rank order,
  * fp32 adds against float64 arithmetic, bf16 rounding against a rational-
  * arithmetic rounder and against torch's CPU cast, hand-derived ties
- * (tests/golden/bf16_ties.txt).  The workload generator below is a definition,
+ * (tests/golden/bf16_ties.txt), and all 2^32 two-rank bf16 pairs against a
+ * binary64 route with a distance-based rounding (tests/golden/pairs_bruteforce.c).  The workload generator below is a definition,
  * not a result: it is pinned by range, moment and frequency checks.
  *
  * Build: gcc -O1 -ffp-contract=off -fno-fast-math -fPIC -shared (see oracle/oracle.py).
