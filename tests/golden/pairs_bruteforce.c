@@ -12,6 +12,10 @@
  * Usage: pairs_bruteforce [first_a last_a]   (default 0 65535).  Prints the number of pairs
  * checked and of mismatches; exit status 1 on any mismatch.  Links against the oracle's C
  * source (test infrastructure only).
+ *
+ *        pairs_bruteforce round first_hi last_hi
+ * checks the oracle's binary32 -> bf16 rounding alone on every bit pattern whose upper 16 bits
+ * lie in [first_hi, last_hi] (all 2^32 patterns for 0 65535) against the same distance rule.
  */
 #include <math.h>
 #include <stdint.h>
@@ -20,6 +24,7 @@
 #include <string.h>
 
 void oracle_allreduce_bf16(const uint16_t *const *x, int P, size_t n, uint16_t *out);
+uint16_t oracle_f32_to_bf16(float f);
 
 static double widen(uint16_t h)
 {
@@ -49,8 +54,29 @@ static uint16_t nearest_bf16(float f)
     return (uint16_t)((((lo_bits >> 16) & 1u) == 0u ? lo_bits : hi_bits) >> 16);   /* tie: even mantissa */
 }
 
+static int check_rounding(unsigned first_hi, unsigned last_hi)
+{
+    unsigned long long checked = 0, bad = 0;
+    for (unsigned hi = first_hi; hi <= last_hi && hi < 65536u; ++hi)
+        for (unsigned lo = 0; lo < 65536u; ++lo) {
+            const uint32_t u = (hi << 16) | lo;
+            float f;
+            memcpy(&f, &u, 4);
+            const uint16_t got = oracle_f32_to_bf16(f), want = nearest_bf16(f);
+            if (got != want) {
+                if (bad < 10) fprintf(stderr, "bits=%08x oracle=%04x expected=%04x\n", u, got, want);
+                ++bad;
+            }
+            ++checked;
+        }
+    printf("%llu %llu\n", checked, bad);
+    return bad ? 1 : 0;
+}
+
 int main(int argc, char **argv)
 {
+    if (argc > 3 && strcmp(argv[1], "round") == 0)
+        return check_rounding((unsigned)strtoul(argv[2], NULL, 0), (unsigned)strtoul(argv[3], NULL, 0));
     const unsigned first = argc > 2 ? (unsigned)strtoul(argv[1], NULL, 0) : 0u;
     const unsigned last = argc > 2 ? (unsigned)strtoul(argv[2], NULL, 0) : 65535u;
     enum { N = 65536 };

@@ -227,7 +227,8 @@ def test_two_rank_bf16_pairs_against_float64_route(oracle):
 
 def test_all_two_rank_bf16_pairs_exhaustively(tmp_path):
     """All 2^32 pairs of bf16 values through the C oracle, against the binary64 route and a distance-based
-    rounding written separately in tests/golden/pairs_bruteforce.c (four processes, a quarter of `a` each)."""
+    rounding written separately in tests/golden/pairs_bruteforce.c (four processes, a quarter of `a` each); and
+    the oracle's binary32 -> bf16 rounding on all 2^32 binary32 bit patterns against the same distance rule."""
     import subprocess
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     flags = ["-std=c11", "-ffp-contract=off", "-fno-fast-math"]
@@ -235,16 +236,17 @@ def test_all_two_rank_bf16_pairs_exhaustively(tmp_path):
     subprocess.check_call(["gcc", "-O1", *flags, "-c", os.path.join(root, "oracle", "sifar_oracle.c"), "-o", o1])
     subprocess.check_call(["gcc", "-O2", *flags, "-c", os.path.join(root, "tests", "golden", "pairs_bruteforce.c"), "-o", o2])
     subprocess.check_call(["gcc", o1, o2, "-lm", "-o", exe])
-    procs = [subprocess.Popen([exe, str(q * 16384), str(q * 16384 + 16383)], stdout=subprocess.PIPE,
-                              stderr=subprocess.PIPE, text=True) for q in range(4)]
-    checked = 0
-    for pr in procs:
-        out, err = pr.communicate(timeout=600)
-        assert pr.returncode == 0, err
-        c, bad = (int(v) for v in out.split())
-        assert bad == 0
-        checked += c
-    assert checked == 1 << 32
+    for mode in ([], ["round"]):          # all pairs of bf16 values; then the rounding alone on all binary32 patterns
+        procs = [subprocess.Popen([exe, *mode, str(q * 16384), str(q * 16384 + 16383)], stdout=subprocess.PIPE,
+                                  stderr=subprocess.PIPE, text=True) for q in range(4)]
+        checked = 0
+        for pr in procs:
+            out, err = pr.communicate(timeout=600)
+            assert pr.returncode == 0, err
+            c, bad = (int(v) for v in out.split())
+            assert bad == 0
+            checked += c
+        assert checked == 1 << 32
 
 
 @pytest.mark.parametrize("P", [3, 5, 8])
