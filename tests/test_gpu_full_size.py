@@ -130,3 +130,24 @@ def test_large_payload_with_late_producers_uses_the_deferring_regime(oracle):
             assert_bits_equal(got, want, BF16, f"mode {mode}")
             st = sf.sifar_get_stats(ctx.h)
             assert st["timeouts"] == 0 and st["calls"] == 1
+
+
+def test_every_pair_of_bf16_values_through_the_gpu(oracle):
+    """P = 2: all 2^32 pairs (a, b) of bf16 bit patterns, 64 calls of 2^26 elements, against the oracle."""
+    n = 1 << 26
+    low = np.tile(np.arange(65536, dtype=np.uint16), n >> 16)                       # b: every value, over and over
+    with Ctx(2, n, BF16) as ctx:
+        xb = to_device(low)
+        out = torch.empty(n, dtype=torch.int16, device="cuda")
+        for chunk in range(64):
+            a = np.repeat(np.arange(chunk << 10, (chunk + 1) << 10, dtype=np.uint32).astype(np.uint16), 65536)
+            xa = to_device(a)
+            mode = (sf.SPECULATIVE, sf.DUALBUF, sf.BARRIER_ONESHOT)[chunk % 3]
+            allreduce_via_pack(ctx, [xa, xb], n, mode, out)
+            torch.cuda.synchronize()
+            assert sf.sifar_status(ctx.h) == 0
+            got = out.cpu().numpy().view(np.uint16)
+            want = oracle.allreduce([a, low], BF16)
+            bad = np.nonzero(got != want)[0]
+            assert bad.size == 0, f"chunk {chunk}: {bad.size} pairs differ, first a={a[bad[0]]:#06x} b={low[bad[0]]:#06x} " \
+                                  f"gpu={got[bad[0]]:#06x} oracle={want[bad[0]]:#06x}"
