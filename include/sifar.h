@@ -27,6 +27,9 @@
  *   SIFAR_POLL_PACE_NS/_MIN sleep between polling rounds above _MIN pairs (0 = unpaced)
  *   SIFAR_POLL_SENTINEL_MIN persistent chain: above this many pairs a warp first waits on one slot per rank (16384)
  *   SIFAR_CHAIN_CLUSTER     0 = persistent chain without thread-block clusters
+ *   SIFAR_CHAIN_PDL         0 = stream / graph chains record the step events the plain way (by default the
+ *                           all-reduce of a step fires its event as soon as all its CTAs have started, and the
+ *                           next step's producers wait inside the kernel for its completion)
  *   SIFAR_PDL               0 = reducers are launched without programmatic dependent launch (read when the
  *                           library is loaded).  By default a reducer with more CTAs than the GPU has SMs
  *                           may become resident while the kernel before it on its stream drains; it reads

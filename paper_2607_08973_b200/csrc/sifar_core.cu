@@ -640,11 +640,25 @@ __global__ void k_set_epoch(DevState *st, uint32_t e) { st->epoch = e; }
  */
 static bool g_pdl = !(getenv("SIFAR_PDL") && atoi(getenv("SIFAR_PDL")) == 0);
 
+static thread_local cudaEvent_t g_programmatic_event = nullptr;   /* set by launch_reduce around the launch */
+
 template <typename K>
 static cudaError_t launch_k(K kernel, int grid, cudaStream_t s, const ReduceArgs &a)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(kThreads); cfg.stream = s;
+    if (g_programmatic_event) {
+        /* The event fires once every CTA has released its dependents (right after the kernel's own dependency
+           wait), so kernels of other streams that wait for it can become resident while this one still runs;
+           they call griddepcontrol.wait before they read anything. */
+        cudaLaunchAttribute ev[1];
+        ev[0].id = cudaLaunchAttributeProgrammaticEvent;
+        ev[0].val.programmaticEvent.event = g_programmatic_event;
+        ev[0].val.programmaticEvent.flags = 0;
+        ev[0].val.programmaticEvent.triggerAtBlockStart = 0;
+        cfg.attrs = ev; cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kernel, a);
+    }
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
@@ -735,9 +749,11 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
     const size_t ntiles = tiles_for(reduce_units(ctx, rl.n, rl.mode), unroll_for(ctx->P));
     a.two_phase = ntiles > (size_t)ctx->sm_count ? 1u : 0u;
     a.janitors = (uint32_t)ctx->sm_count;
+    g_programmatic_event = rl.programmatic_event;
     cudaError_t err = (ctx->dtype == SIFAR_BF16)
         ? launch_reduce_dt<SIFAR_BF16>(ctx->P, rl.mode, (int)ntiles, stream, a)
         : launch_reduce_dt<SIFAR_F32>(ctx->P, rl.mode, (int)ntiles, stream, a);
+    g_programmatic_event = nullptr;
     SIFAR_CUDA(err);
     return SIFAR_OK;
 }

@@ -118,6 +118,7 @@ struct ReduceLaunch {
     size_t n;
     int mode;
     uint32_t parity;                 /* parity the host expects the call number to have */
+    cudaEvent_t programmatic_event;  /* NULL, or an event the kernel fires as soon as all its CTAs have started */
 };
 
 int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream);
