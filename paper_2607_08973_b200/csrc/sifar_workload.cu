@@ -57,7 +57,36 @@ template <int DT, int MODE>
 __global__ void __launch_bounds__(kProdThreads) k_produce(const ProduceArgs a)
 {
     DevState *st = a.st;
-    __shared__ uint32_t s_e, s_t;
+    __shared__ uint32_t s_e, s_t, s_guess;
+    constexpr int NW = (MODE == SIFAR_SPECULATIVE) ? 3 : 4;
+    constexpr int EPU = NW * ((DT == SIFAR_BF16) ? 2 : 1);
+    const size_t tid = (size_t)blockIdx.x * kProdThreads + threadIdx.x;
+    const size_t nthreads = (size_t)gridDim.x * kProdThreads;
+    /*
+     * The kernel may be resident before the all-reduce it follows has finished (that all-reduce fires the step's
+     * event as soon as its CTAs have started).  The step number is known even then: the call number read now is
+     * the previous call's or the one before it, and the parity of this call is fixed at launch.  So the seeded
+     * half of the thread's first unit is computed ahead of the dependency wait, as in the persistent kernel.
+     */
+    if (threadIdx.x == 0) {
+        uint32_t tg = a.t_fixed;
+        if (MODE != kModeNoAllreduce) {
+            const uint32_t seen = ld_relaxed_u32(&st->epoch);
+            tg = (((seen + 1u) & 1u) == a.parity ? seen + 1u : seen + 2u) - a.base_epoch;
+        }
+        s_guess = tg;
+    }
+    __syncthreads();
+    const uint32_t t_ahead = s_guess;
+    float z0[EPU];
+    {
+        const Gen g0 = make_gen(a.w, a.rank, t_ahead);
+        if (tid * EPU < (size_t)a.n) {
+            unit_noise<DT, NW>(g0, t_ahead == 1u, tid * EPU, (size_t)a.n, z0);
+#pragma unroll
+            for (int k = 0; k < EPU; ++k) asm volatile("" : "+f"(z0[k]));     /* keep it above the wait */
+        }
+    }
     /* if the all-reduce before this operation released its dependents early, wait here for its completion */
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (threadIdx.x == 0) {
@@ -90,22 +119,23 @@ __global__ void __launch_bounds__(kProdThreads) k_produce(const ProduceArgs a)
     const Gen g = make_gen(a.w, a.rank, t);
     const bool first = (t == 1u);
     const size_t n = (size_t)a.n;
-    const size_t tid = (size_t)blockIdx.x * kProdThreads + threadIdx.x;
-    const size_t nthreads = (size_t)gridDim.x * kProdThreads;
-    if (MODE == SIFAR_SPECULATIVE) {
-        constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;
+    const bool ahead_ok = (t == t_ahead);              /* always, unless the context was used against its contract */
+    if constexpr (MODE == SIFAR_SPECULATIVE) {
+        constexpr int EPS = EPU;
         const size_t nslots = (n + EPS - 1) / EPS;
         for (size_t s = tid; s < nslots; s += nthreads) {
             uint32_t w[3];
-            produce_words<DT, 3>(g, first, a.prev, s * EPS, n, w);
+            if (s == tid && ahead_ok) unit_combine<DT, 3>(g, first, a.prev, s * EPS, n, z0, w);
+            else produce_words<DT, 3>(g, first, a.prev, s * EPS, n, w);
             store_slot(reinterpret_cast<uint4 *>(a.dst), s, w[0], w[1], w[2], e);
         }
     } else {
-        constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
+        constexpr int EPV = EPU;
         const size_t nvec = (n + EPV - 1) / EPV;       /* the last vector is zero-padded inside the context's buffer */
         for (size_t v = tid; v < nvec; v += nthreads) {
             uint32_t w[4];
-            produce_words<DT, 4>(g, first, a.prev, v * EPV, n, w);
+            if (v == tid && ahead_ok) unit_combine<DT, 4>(g, first, a.prev, v * EPV, n, z0, w);
+            else produce_words<DT, 4>(g, first, a.prev, v * EPV, n, w);
             st_slot(reinterpret_cast<uint4 *>(a.dst) + v, make_uint4(w[0], w[1], w[2], w[3]));
         }
         if (MODE != kModeNoAllreduce)
