@@ -226,13 +226,15 @@ def measure_modes(sf, torch, synth, n, warmup, reps, impls, modes, rounds=3, nam
     return res
 
 
-def measure_roofline(sf, torch, P_, n, mode, warmup, iters, dtype=0, nctx=6):
+def measure_roofline(sf, torch, P_, n, mode, warmup, iters, dtype=0, nctx=24):
     """Device time per launch of the reducer kernel on payloads larger than L2.
 
-    `nctx` contexts are packed (untimed), then their reducers run back to back between two CUDA events on
-    the launching stream; every launch reads partials that five other launches' traffic (each larger
-    than the 126 MB L2) has since evicted.  A spin kernel ahead of the first event lets the host enqueue the
-    whole batch before the device reaches it, so host launch cost is not in the timed region.
+    `nctx` contexts are packed (untimed; every rank on its own producer stream, as in the protocol), then
+    their reducers run back to back between two CUDA events on the launching stream; every launch reads
+    partials that the other launches' traffic (each larger than the 126 MB L2) has since evicted.  A spin
+    kernel ahead of the first event lets the host enqueue the whole batch before the device reaches it, so
+    host launch cost is not in the timed region.  A pair of events costs about 13 us of its own (start and
+    drain of the first and last kernel); with 24 launches in between that is 0.5 us per launch.
     """
     td = torch.int16 if dtype == 0 else torch.float32
     ctxs = [sf.sifar_create(P_, n, dtype) for _ in range(nctx)]
@@ -240,21 +242,26 @@ def measure_roofline(sf, torch, P_, n, mode, warmup, iters, dtype=0, nctx=6):
           else torch.randn(n, device="cuda") for _ in range(P_)]
     outs = [torch.empty(n, dtype=td, device="cuda") for _ in range(2)]
     s = torch.cuda.Stream()
+    ps = [torch.cuda.Stream() for _ in range(P_)]
+    torch.cuda.synchronize()
     times = []
-    with torch.cuda.stream(s):
-        for it in range(warmup + iters):
-            for h in ctxs:
-                for r in range(P_):
-                    sf.sifar_pack(h, r, xs[r].data_ptr(), n, mode, s.cuda_stream)
-            sf.sifar_spin(2_000_000, s.cuda_stream)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(s)
-            for i, h in enumerate(ctxs):
-                sf.sifar_allreduce(h, None, outs[i & 1].data_ptr(), n, mode, s.cuda_stream)
-            b.record(s)
-            s.synchronize()
-            if it >= warmup:
-                times.append(a.elapsed_time(b) * 1e-3 / nctx)
+    for it in range(warmup + iters):
+        for h in ctxs:
+            for r in range(P_):
+                sf.sifar_pack(h, r, xs[r].data_ptr(), n, mode, ps[r].cuda_stream)
+        for r in range(P_):
+            s.wait_stream(ps[r])
+        sf.sifar_spin(2_000_000, s.cuda_stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(s)
+        for i, h in enumerate(ctxs):
+            sf.sifar_allreduce(h, None, outs[i & 1].data_ptr(), n, mode, s.cuda_stream)
+        b.record(s)
+        s.synchronize()
+        for r in range(P_):
+            ps[r].wait_stream(s)
+        if it >= warmup:
+            times.append(a.elapsed_time(b) * 1e-3 / nctx)
     status = [sf.sifar_status(h) for h in ctxs]
     for h in ctxs:
         sf.sifar_destroy(h)
@@ -328,10 +335,7 @@ def payload_sweep(sf, torch, exps=range(10, 26), ranks=(2, 4, 8)):
                     mean_s, med_s, _ = measure_roofline(sf, torch, P_, n, mode, 2, 5, dtype=dtype, nctx=nctx)
                     alg = sf.sifar_algorithmic_bytes(P_, dtype, n, mode)
                     row[sf.MODE_NAMES[mode]] = {"us": round(med_s * 1e6, 2), "GBps": round(alg / med_s / 1e9, 1)}
-                # the size-adaptive choice between the two barrier-free modes, and what it costs against the better one
-                pick = sf.MODE_NAMES[sf.sifar_mode_for_payload(P_, dtype, n)]
-                best = min(row["dualbuf"]["us"], row["speculative"]["us"])
-                row["adaptive"] = {"mode": pick, "us": row[pick]["us"], "over_best_pct": round(100 * (row[pick]["us"] / best - 1), 1)}
+                row["speculative"]["format"] = "tiles" if sf.sifar_spec_format(P_, dtype, n) == sf.FORMAT_TILES else "slots"
                 rows.append(row)
     return rows
 
@@ -367,7 +371,7 @@ def measure_symmetric(sf, torch, synth, ranks, n, name="llama", steps=ARS_PER_ST
 
 
 def retry_overhead(sf, torch, synth, ranks=(2, 4, 8), kbytes=(8, 16, 32), forced=(0, 1, 2, 3)):
-    """Section 7, "Retry Overhead": p50 per all-reduce of the persistent chain with a fixed number of
+    """Section 6.3, "Retry Overhead": p50 per all-reduce of the persistent chain with a fixed number of
     forced retries, next to the barrier baseline of the same chain."""
     res = {}
     for P_ in ranks:

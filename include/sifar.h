@@ -80,18 +80,53 @@ typedef enum {
 enum { SIFAR_MAX_RANKS = 8 };
 
 /*
+ * ORDERING CONTRACT (what the caller's streams must guarantee; it is the co-design
+ * the paper asks of the inference engine, Sections 3.3 and 4.2 "Dual Buffering":
+ * the input of an all-reduce is the output of the operation before it).
+ *   - The producer of call e + 1 for any rank (sifar_pack, sifar_arrive,
+ *     sifar_wait_writable, or a caller's own kernel writing into the buffer that
+ *     sifar_rank_buffer returned) must be ORDERED AFTER the reducer kernel of call
+ *     e: same stream, an event, or a graph edge.  In a decode step it is anyway,
+ *     because it consumes `out` of call e.  The producer kernels take the call
+ *     number from device memory when they run (so that a replayed CUDA graph needs
+ *     no new arguments), and the reducer advances it when its last CTA is done.  A
+ *     producer that runs before that finds the number one short; it is detected by
+ *     the number's parity and the context turns SIFAR_ERR_EPOCH (sticky), in every
+ *     mode, instead of overwriting a buffer under a running reducer.
+ *   - The producer of call e must NOT be ordered before the reducer of call e by
+ *     anything but the mode's own flags or tags: that wait is the thing measured.
+ *   - sifar_allreduce calls on one context are enqueued on one stream (or otherwise
+ *     serialized).  A reducer's reads are ordered by the protocol alone, its writes
+ *     (`out`, the call number) by the stream: a large reducer whose producers were
+ *     enqueued on other streams starts polling and loading while the kernel before
+ *     it on its stream still drains, and stores only when that kernel is complete.
+ *   - BARRIER_ONESHOT: the device-side bottom barrier (done flags, and the wait for
+ *     them in sifar_pack / sifar_wait_writable) protects the single buffer against
+ *     a producer that is ordered after the reducer's START only, as a fused
+ *     forward-pass kernel would be.  With whole kernels in stream order the wait is
+ *     already satisfied when the producer runs; the baseline then pays the
+ *     reducer-side half only (all CTAs counted, P flag stores).
+ */
+
+/*
  * Create a context for P ranks (1..8) of at most max_elems elements of `dtype`
- * on the CURRENT device.  Allocates (cudaMalloc), once, per rank: two plain
+ * on the CURRENT device.  The operation is the oneshot all-reduce of Section 3.1;
+ * the two parity sets of rank buffers it allocates are the buffer-ownership side
+ * of dual buffering (Section 4.2, "Dual Buffering": the previous input buffer must
+ * stay alive until the next all-reduce has run).  Allocates (cudaMalloc), once, per rank: two plain
  * buffers, two slot buffers, and the shared flag / call-number / status words;
  * everything zero-filled, so every tag starts as 0 = "never valid".
  * Synchronizes the device.  Returns NULL on failure (see sifar_last_error()).
  */
 sifar_ctx *sifar_create(int P, size_t max_elems, int dtype);
 
-/* Waits for the context's outstanding work, frees everything.  NULL is a no-op. */
+/* Waits for the context's outstanding work, frees everything (the buffers of Section 4.2, "Dual Buffering",
+   live exactly as long as the context).  NULL is a no-op. */
 int sifar_destroy(sifar_ctx *ctx);
 
 /*
+ * The all-reduce (Section 3.1 "Oneshot": pull all P partials, reduce locally; with
+ * the barriers of `mode`, Sections 3.3, 3.5 and 4.2).
  * Enqueue call number e = (calls so far) + 1 on `stream`: one reducer kernel, no
  * allocation, no host synchronization.
  *
@@ -144,7 +179,9 @@ int sifar_allreduce_host(sifar_ctx *ctx, const void *const *host_rank_ptrs, void
  * `mode`.  *ptr: device buffer (plain elements for the barrier modes; 16-byte
  * slots {12 data bytes, 4-byte little-endian tag} for SPECULATIVE, slot i holding
  * elements [i*k, i*k+k), k = 6 for bf16 and 3 for fp32, a short last slot padded
- * with zeros).  *epoch: the call number, i.e. the tag value.  Either may be NULL.
+ * with zeros; plain elements in the large-payload format, see sifar_spec_format).
+ * *epoch: the call number, i.e. the tag value.  Either may be NULL.  The kernel that
+ * writes there follows the ordering contract above.
  */
 int sifar_rank_buffer(sifar_ctx *ctx, int rank, int mode, void **ptr, unsigned *epoch);
 
@@ -153,21 +190,25 @@ int sifar_rank_buffer(sifar_ctx *ctx, int rank, int mode, void **ptr, unsigned *
  * plain elements from `src` (device, 16-byte aligned) into the context's buffer
  * of `rank` for the NEXT call: a copy followed by a release of the rank's arrival
  * flag (barrier modes; BARRIER_ONESHOT first waits for the rank's done flag of
- * the previous call), or tagged 16-byte slot stores and nothing else (SPECULATIVE).
+ * the previous call), or tagged 16-byte slot stores and nothing else (SPECULATIVE;
+ * plain stores and one flag per 16 KiB block in its large-payload format, see
+ * sifar_spec_format).  Must be ordered after the previous call's reducer (ordering
+ * contract above); a kernel that was not turns the context SIFAR_ERR_EPOCH.
  */
 int sifar_pack(sifar_ctx *ctx, int rank, const void *src, size_t n, int mode, void *stream);
 
 /*
  * Barrier modes with partials written by the caller's own kernels: enqueue on
  * `stream` (after those kernels) the release of `rank`'s arrival flag for the
- * NEXT call.
+ * NEXT call.  Same ordering contract as sifar_pack.
  */
 int sifar_arrive(sifar_ctx *ctx, int rank, int mode, void *stream);
 
 /*
  * BARRIER_ONESHOT only: enqueue on `stream` the producer-side half of the bottom
  * barrier, a bounded wait until the reducer of the previous call has released
- * `rank`'s done flag.  Enqueue it before the kernel that overwrites the buffer.
+ * `rank`'s done flag.  Enqueue it before the kernel that overwrites the buffer,
+ * and after the previous call's reducer in stream or event order (ordering contract).
  */
 int sifar_wait_writable(sifar_ctx *ctx, int rank, void *stream);
 
@@ -196,19 +237,38 @@ int sifar_reset(sifar_ctx *ctx, void *stream);
 int sifar_debug_set_epoch(sifar_ctx *ctx, unsigned calls_so_far);
 
 /*
- * Size-adaptive choice between the two barrier-free modes.  The paper has no
- * counterpart: it targets decode payloads of 8-32 KB (Section 5), where the tags
- * of the speculative slots cost nothing that matters.  For large payloads the
+ * The two layouts in which a partial travels in SIFAR_SPECULATIVE, chosen by size.
+ * The paper has no counterpart: it targets decode payloads of 8-32 KB (Section 5),
+ * where the tags of the slots cost nothing that matters.  For large payloads the
  * tagged slots move a third more bytes than plain data, which is what bounds the
- * reducer there.  Returns SIFAR_SPECULATIVE while all P partials together stay
- * below 16 MiB (the crossover measured on B200 for P = 2, 4 and 8, bf16 and fp32:
- * 2 MiB per rank at P = 8, 8 MiB per rank at P = 2) and SIFAR_DUALBUF from there
- * on; SIFAR_ERR_INVALID for a bad P or dtype.  Pure function, no device access.
+ * reducer there, so from 16 MiB for all P partials together the speculative mode
+ * keeps the early start (Section 3.5) but validates per block instead of per slot:
+ *
+ * SIFAR_FORMAT_SLOTS   16-byte slots {12 data bytes, 4-byte tag}; no flag at all.
+ * SIFAR_FORMAT_TILES   plain elements at the start of the same rank buffer, plus one
+ *                      arrival flag per block of 16 KiB (8192 bf16 / 4096 fp32
+ *                      elements; the last block may be short), set to the call number
+ *                      with release semantics once the block is stored.  A reducer CTA
+ *                      acquires only the P flags of the block its tile lies in, so
+ *                      tiles are reduced as they land; there is no call-wide barrier
+ *                      and no tag traffic.
+ *
+ * sifar_spec_format() is a pure function (no device access): the format that
+ * sifar_pack() and sifar_allreduce() use for n elements per rank; SIFAR_ERR_INVALID
+ * for a bad P or dtype.  sifar_tile_flags(): where `rank`'s block flags of the NEXT
+ * call lie, for producers that store their partial themselves (device helper
+ * sifar::signal_block in sifar_device.cuh): *flags = device address of the rank's
+ * flag of block 0, a 32-bit word; the flag of block b is stride_words words further
+ * per block (the P ranks' flags of one block share a 32-byte sector, so a reducer
+ * CTA fetches them with one access); block b = elements [b * elems_per_flag,
+ * (b + 1) * elems_per_flag).  Any of the three results may be NULL.
  */
-int sifar_mode_for_payload(int P, int dtype, size_t n);
+typedef enum { SIFAR_FORMAT_SLOTS = 0, SIFAR_FORMAT_TILES = 1 } sifar_format;
+int sifar_spec_format(int P, int dtype, size_t n);
+int sifar_tile_flags(sifar_ctx *ctx, int rank, void **flags, size_t *elems_per_flag, size_t *stride_words);
 
 /*
- * Measurement hook for the retry-latency experiment (Section 7, "Retry Overhead":
+ * Measurement hook for the retry-latency experiment (Section 6.3, "Retry Overhead":
  * latency of the no-retry case and what each further retry adds, obtained by
  * forcing a fixed number of retries).  With rounds = k > 0 the speculative reducer
  * treats the attempt that found all P copies of a slot valid as mis-speculated,
@@ -251,6 +311,13 @@ int sifar_debug_force_retries(sifar_ctx *ctx, unsigned rounds);
  */
 int sifar_allreduce_noalloc(const void *const *rank_ptrs, int P, void *out, size_t n, int dtype, void *stream);
 size_t sifar_noalloc_max_elems(void);
+/*
+ * The bookkeeping words of the current device's array, for tests and diagnosis (waits for the device, copies
+ * to the caller's array, allocates nothing): out[0] = count of finished CTAs (0 between calls: the last CTA of
+ * a call re-arms it), out[1] = calls completed on this device since the library was loaded, out[2] = n of the
+ * last completed call.
+ */
+int sifar_noalloc_counters(unsigned long long out[3]);
 
 /* Geometry helpers (no device work). */
 size_t sifar_slot_count(int dtype, size_t n);          /* slots needed for n elements  */

@@ -139,6 +139,17 @@ __device__ __forceinline__ void signal_arrival(uint32_t *counter, uint32_t nctas
     }
 }
 
+/*
+ * Arrival of one block of the flagged-tile format (speculative mode, large payloads; see
+ * sifar_spec_format() and sifar_tile_flags()).  Every thread of the CTA that stored the block calls this
+ * after its last store of the block; one thread releases the block's flag.
+ */
+__device__ __forceinline__ void signal_block(uint32_t *flags, size_t stride_words, size_t block, uint32_t epoch)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) st_release_u32(flags + block * stride_words, epoch);
+}
+
 /* bf16 pair <-> binary32 (the low half of a word is the element with the lower index). */
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }

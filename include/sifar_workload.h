@@ -68,7 +68,7 @@ typedef enum {
 } sifar_chain_impl;
 
 /* Fourth "mode", chains only: no all-reduce at all; each rank's next operation consumes its own
-   partial (the paper's "feed the input of the all-reduce to the next operation" experiment, Section 2.3).
+   partial (the paper's "feed the input of the all-reduce to the next operation" experiment, Section 2.4).
    A timing floor; its results are not a sum. */
 enum { SIFAR_CHAIN_NO_ALLREDUCE = 3 };
 
@@ -169,7 +169,8 @@ int sifar_symchain_run(sifar_symchain *chain, void *stream);
 int sifar_symchain_stamps(sifar_symchain *chain, unsigned long long *stamps);
 int sifar_symchain_rank_stamps(sifar_symchain *chain, int rank, unsigned long long *stamps);
 /*
- * Mis-speculation per rank (Section 7: the fraction of all-reduces that retried):
+ * Mis-speculation per rank (Section 6.3, "Mis-Speculation and Verification Overhead": the
+ * fraction of all-reduces that retried):
  * host_per_rank[r] = number of steps so far in which rank r had to load a slot
  * again, r = 0..P-1 (speculative mode; zeros otherwise).  Synchronizes.  The
  * context's statistics count a step as a call with retry if any rank retried.
@@ -189,10 +190,38 @@ int sifar_workload_next(const sifar_workload *w, int rank, unsigned t, int dtype
 int sifar_workload_delays(const sifar_workload *w, int P, unsigned t, unsigned *host_out);
 
 /*
+ * Loads the code of the helper and producer kernels of this library on the current
+ * device.  With lazy module loading (the CUDA default) the first launch of a kernel
+ * loads it, and that load can wait until the device is idle: a helper launched for
+ * the first time while a reducer already polls for its data would block the host
+ * until that reducer gave up.  Call once before scripting such orderings (the
+ * Python binding does when it loads the library on a machine with a GPU; chain
+ * creation does for what a chain launches).  Kernels of sifar.h are loaded by
+ * sifar_create.
+ */
+int sifar_workload_preload(void);
+
+/*
  * Enqueue a kernel that busy-waits `ns` nanoseconds (at most 50 ms) on `stream`:
  * used to force producer / reducer orderings in tests and benchmarks.
  */
 int sifar_spin(unsigned ns, void *stream);
+
+/*
+ * Stand-ins for a caller's own fused producer (tests): store a part of a rank's
+ * partial for call number `tag` with the device helpers of sifar_device.cuh, on
+ * `stream`.  src: n plain elements (device, 16-byte aligned).
+ * sifar_store_slots:  slots [first_slot, first_slot + nslots) of the tagged-slot
+ *                     format into `slots` (the pointer sifar_rank_buffer() returned).
+ * sifar_store_blocks: blocks [first_block, first_block + nblocks) of the flagged-tile
+ *                     format as plain elements into `dst` (the same pointer), each
+ *                     followed by the release of its flag; flags / stride_words as
+ *                     returned by sifar_tile_flags().
+ */
+int sifar_store_slots(const void *src, void *slots, size_t first_slot, size_t nslots, size_t n, int dtype,
+                      unsigned tag, void *stream);
+int sifar_store_blocks(const void *src, void *dst, void *flags, size_t stride_words, size_t first_block,
+                       size_t nblocks, size_t n, int dtype, unsigned tag, void *stream);
 
 /*
  * 16-byte access atomicity check (the speculative slots rely on it): `writers`

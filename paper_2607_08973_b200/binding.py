@@ -1,4 +1,5 @@
-"""Thin ctypes binding of ``libsifar.so``: same names as ``include/sifar.h``.
+"""Thin ctypes binding of ``libsifar.so`` (``include/sifar.h``) and of
+``libsifar_bench.so`` (``include/sifar_workload.h``): same names as the headers.
 
 Argument marshalling only.  Every step of the all-reduce runs in the CUDA
 library; there is no CPU fallback: if the library has not been built, the first
@@ -14,9 +15,12 @@ BF16, F32 = 0, 1
 BARRIER_ONESHOT, DUALBUF, SPECULATIVE = 0, 1, 2
 OK, ERR_INVALID, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT, ERR_EPOCH = 0, -1, -2, -3, -4, -5
 MODE_NAMES = {BARRIER_ONESHOT: "barrier_oneshot", DUALBUF: "dualbuf", SPECULATIVE: "speculative"}
+FORMAT_SLOTS, FORMAT_TILES = 0, 1
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsifar.so")
+_BENCH_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsifar_bench.so")
 _lib = None
+_bench_lib = None
 
 
 class SifarError(RuntimeError):
@@ -50,12 +54,14 @@ def lib() -> ctypes.CDLL:
             "sifar_reset": (ci, [vp, vp]),
             "sifar_debug_set_epoch": (ci, [vp, cu]),
             "sifar_debug_force_retries": (ci, [vp, cu]),
-            "sifar_mode_for_payload": (ci, [ci, ci, sz]),
+            "sifar_spec_format": (ci, [ci, ci, sz]),
+            "sifar_tile_flags": (ci, [vp, ci, ctypes.POINTER(vp), ctypes.POINTER(sz), ctypes.POINTER(sz)]),
             "sifar_slot_count": (sz, [ci, sz]),
             "sifar_algorithmic_bytes": (sz, [ci, ci, sz, ci]),
             "sifar_last_error": (ctypes.c_char_p, []),
             "sifar_allreduce_noalloc": (ci, [vp, ci, vp, sz, ci, vp]),
             "sifar_noalloc_max_elems": (sz, []),
+            "sifar_noalloc_counters": (ci, [ctypes.POINTER(ctypes.c_ulonglong)]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -140,11 +146,18 @@ def sifar_debug_set_epoch(ctx: int, calls_so_far: int) -> int:
     return _check(lib().sifar_debug_set_epoch(ctx, calls_so_far))
 
 
-def sifar_mode_for_payload(P: int, dtype: int, n: int) -> int:
-    mode = lib().sifar_mode_for_payload(P, dtype, n)
-    if mode < 0:
-        raise SifarError(mode, sifar_last_error())
-    return mode
+def sifar_spec_format(P: int, dtype: int, n: int) -> int:
+    fmt = lib().sifar_spec_format(P, dtype, n)
+    if fmt < 0:
+        raise SifarError(fmt, sifar_last_error())
+    return fmt
+
+
+def sifar_tile_flags(ctx: int, rank: int) -> tuple[int, int, int]:
+    """(device address of the rank's flag of block 0, elements per flag, words between two blocks' flags)."""
+    p, k, st = ctypes.c_void_p(), ctypes.c_size_t(), ctypes.c_size_t()
+    _check(lib().sifar_tile_flags(ctx, rank, ctypes.byref(p), ctypes.byref(k), ctypes.byref(st)))
+    return (p.value or 0), k.value, st.value
 
 
 def sifar_debug_force_retries(ctx: int, rounds: int) -> int:
@@ -168,8 +181,14 @@ def sifar_noalloc_max_elems() -> int:
     return lib().sifar_noalloc_max_elems()
 
 
+def sifar_noalloc_counters() -> dict:
+    buf = (ctypes.c_ulonglong * 3)()
+    _check(lib().sifar_noalloc_counters(buf))
+    return {"cta_arrive": int(buf[0]), "calls": int(buf[1]), "elements": int(buf[2])}
+
+
 # ---------------------------------------------------------------------------
-# include/sifar_workload.h: synthetic decode-step chains
+# include/sifar_workload.h (libsifar_bench.so): synthetic decode-step chains
 # ---------------------------------------------------------------------------
 CHAIN_STREAMS, CHAIN_GRAPH, CHAIN_PERSISTENT = 0, 1, 2
 CHAIN_NO_ALLREDUCE = 3
@@ -187,13 +206,16 @@ def make_workload(kind: int, seed: int, scale: float, sigma: float, outlier_mod:
     return sifar_workload(kind, seed, scale, sigma, outlier_mod, delay_max_ns)
 
 
-_wl_ready = False
-
-
 def _wl() -> ctypes.CDLL:
-    global _wl_ready
-    L = lib()
-    if not _wl_ready:
+    """Load the workload library (once); it links against libsifar.so, which is loaded first."""
+    global _bench_lib
+    if _bench_lib is None:
+        lib()
+        if not os.path.exists(_BENCH_LIB_PATH):
+            raise RuntimeError(
+                f"{_BENCH_LIB_PATH} not found: build it with `python -m paper_2607_08973_b200.build`; "
+                "there is no CPU fallback")
+        L = ctypes.CDLL(_BENCH_LIB_PATH)
         vp, sz, ci, cu = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint
         wp = ctypes.POINTER(sifar_workload)
         ullp = ctypes.POINTER(ctypes.c_ulonglong)
@@ -218,12 +240,20 @@ def _wl() -> ctypes.CDLL:
             "sifar_workload_delays": (ci, [wp, ci, cu, ctypes.POINTER(cu)]),
             "sifar_spin": (ci, [cu, vp]),
             "sifar_tear_check": (ci, [cu, cu, ullp, ullp]),
+            "sifar_workload_preload": (ci, []),
+            "sifar_store_slots": (ci, [vp, vp, sz, sz, sz, ci, cu, vp]),
+            "sifar_store_blocks": (ci, [vp, vp, vp, sz, sz, sz, sz, ci, cu, vp]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
             fn.restype, fn.argtypes = res, args
-        _wl_ready = True
-    return L
+        _bench_lib = L
+    return _bench_lib
+
+
+def sifar_workload_preload() -> int:
+    """Loads the helper kernels' code now, so that no later first launch has to wait for an idle device."""
+    return _check(_wl().sifar_workload_preload())
 
 
 def sifar_chain_ring_stride(dtype: int, n: int) -> int:
@@ -333,3 +363,13 @@ def sifar_tear_check(nslots: int, rounds: int) -> tuple[int, int]:
     torn, reads = ctypes.c_ulonglong(), ctypes.c_ulonglong()
     _check(_wl().sifar_tear_check(nslots, rounds, ctypes.byref(torn), ctypes.byref(reads)))
     return torn.value, reads.value
+
+
+def sifar_store_slots(src: int, slots: int, first_slot: int, nslots: int, n: int, dtype: int, tag: int,
+                      stream: int = 0) -> int:
+    return _check(_wl().sifar_store_slots(src, slots, first_slot, nslots, n, dtype, tag, stream))
+
+
+def sifar_store_blocks(src: int, dst: int, flags: int, stride_words: int, first_block: int, nblocks: int, n: int,
+                       dtype: int, tag: int, stream: int = 0) -> int:
+    return _check(_wl().sifar_store_blocks(src, dst, flags, stride_words, first_block, nblocks, n, dtype, tag, stream))

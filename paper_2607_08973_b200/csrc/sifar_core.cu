@@ -16,6 +16,19 @@
  *   SPECULATIVE      producer r : one 16-byte store {12 B data, tag = e} per slot.
  *                    reducer    : load all P slots at once, accept tag == e,
  *                                 re-load only the stale ones (bounded); sum; store.
+ *     large payloads (flagged tiles): the tags would cost a third more traffic, so
+ *                    producer r : plain stores; one arrival flag = e per 16 KiB block,
+ *                                 released as soon as that block is stored.
+ *                    reducer    : a CTA acquires the P flags of its own tile only,
+ *                                 then loads, sums, stores: tiles are reduced as
+ *                                 they land, there is no call-wide barrier.
+ *
+ * What orders a reducer.  Its READS are ordered by the protocol alone (arrival
+ * flags with release/acquire, or tags inside the slots), never by the stream: a
+ * reducer launched with programmatic stream serialization polls and loads while
+ * the kernel before it on its stream is still draining.  Its WRITES (the result,
+ * the CTA count, the call number) wait for that kernel (griddepcontrol.wait), so
+ * the stream order of results is what the caller expects.
  *
  * The call number lives in device memory (DevState::epoch) and is read by every
  * kernel at entry, so a replayed CUDA graph advances it without new arguments.
@@ -69,6 +82,12 @@ struct ReduceArgs {
     uint32_t janitors;       /* G: how many of the last CTAs sweep up the deferred tiles              */
     unsigned long long spin_ns;
     uint32_t *defer;         /* [0] = number of queued tiles, [1..] = their indices */
+    /* arrival flags a CTA waits for before it loads plain partials: rank r's flag of tile t is
+       flags[(t >> flag_shift) * kFlagStride + r] (one flag per rank and call: flag_shift = 31) */
+    const uint32_t *flags;
+    uint32_t flag_shift;
+    uint32_t early;          /* 1: reads do not wait for the stream's previous kernel, writes do     */
+    uint32_t e_host;         /* the call number the host expects, or 0: take it from device memory   */
 };
 
 struct PackArgs {
@@ -81,7 +100,14 @@ struct PackArgs {
     uint32_t rank;
     uint32_t parity;
     uint32_t wait_delta;     /* 0: no bottom-barrier wait; d: wait for done[rank] >= e - d */
+    uint32_t *tile_flags;    /* flagged-tile format: the flag array of this call's parity ([block][kFlagStride]) */
 };
+
+/* Internal fourth mode of the plain reducer and of the pack kernel: SPECULATIVE in the flagged-tile format. */
+constexpr int kModeTiles = 3;
+
+__device__ __forceinline__ void gdc_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void gdc_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 
 constexpr int kThreads = 256;
 
@@ -97,8 +123,9 @@ constexpr int kThreads = 256;
 template <int MODE>
 __device__ __forceinline__ void publish_call(DevState *st, uint32_t e, int P)
 {
+    st_relaxed_u32(&st->cta_arrive[(e + 1u) & 1u], 0u);               /* re-arm the next call's count (see DevState) */
     atomicAdd(&st->stats[kStatCalls], 1ull);                          /* result unused: fire and forget */
-    if (MODE == SIFAR_SPECULATIVE && ld_relaxed_u32(&st->retry_epoch) == e)
+    if ((MODE == SIFAR_SPECULATIVE || MODE == kModeTiles) && ld_relaxed_u32(&st->retry_epoch) == e)
         atomicAdd(&st->stats[kStatCallsWithRetry], 1ull);
     if (MODE == SIFAR_BARRIER_ONESHOT) {
         /* one fence, then the P done flags: P release stores in a row would each wait for the one before */
@@ -118,7 +145,7 @@ __device__ __forceinline__ void publish_call(DevState *st, uint32_t e, int P)
  * 16-byte loads before the first add.
  */
 template <int DT, int P>
-__device__ __forceinline__ void tile_plain(const ReduceArgs &a, size_t tile, size_t ntiles)
+__device__ __forceinline__ void tile_plain(const ReduceArgs &a, size_t tile, size_t ntiles, bool wait_before_stores)
 {
     constexpr int U = Unroll<P>::value;
     constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;       /* elements per 16-byte vector */
@@ -134,6 +161,7 @@ __device__ __forceinline__ void tile_plain(const ReduceArgs &a, size_t tile, siz
             for (int r = 0; r < P; ++r) x[u][r] = ld_slot(a.src[r] + v);
         }
     }
+    if (wait_before_stores) gdc_wait();                    /* the loads are in flight; nothing was written yet */
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const size_t v = base + (size_t)u * kThreads;
@@ -186,6 +214,8 @@ __host__ __device__ inline size_t tiles_for(size_t units, int per_thread)
     return t ? t : 1;
 }
 
+constexpr uint32_t kQueuedBit = 0x80000000u;      /* in the CTA count: some CTA has queued its tile */
+
 /* Call number, status and parity check at kernel entry.  Returns 0 if the kernel must not run. */
 __device__ __forceinline__ uint32_t entry_epoch(const ReduceArgs &a, uint2 es)
 {
@@ -199,32 +229,95 @@ __device__ __forceinline__ uint32_t entry_epoch(const ReduceArgs &a, uint2 es)
 }
 
 /*
- * Top barrier (Section 3.1, phase 1) by warp 0: the P arrival flags of this call.
- * Returns the call number, or 0 with `give_up` telling why: 1 = not arrived
- * within limit_ns, 2 = error / context dead.
+ * An early reducer may find the call number one short: the kernel before it on its stream is this
+ * context's previous reducer and has not published yet.  Then, and only then, the parity is off by one.
  */
-template <int P>
-__device__ __forceinline__ uint32_t top_barrier(const ReduceArgs &a, unsigned long long limit_ns, int &give_up)
+__device__ __forceinline__ bool predecessor_unpublished(const ReduceArgs &a, uint2 es)
+{
+    return a.early && es.y == 0u && ((es.x + 1u) & 1u) != a.parity;
+}
+
+/*
+ * Top barrier (Section 3.1, phase 1) by warp 0: lane r < P loads rank r's arrival flag of this tile
+ * (acquire).  The flag is the rank's single arrival flag of the call (barrier modes) or the flag of the
+ * 16 KiB block the tile lies in (flagged tiles).
+ *
+ * Fast path: the host passed the call number it expects (a.e_host) and all P flags carry it: one load
+ * per lane, one line, one round trip through the L2, nothing else is touched.  (Every word that each
+ * CTA of a large grid reads is a hot spot in its L2 slice: the call-number line and the CTA-count line
+ * cost 0.6 and 0.35 us per 16 MiB call when every CTA read them.)
+ * Slow path (flags not there yet, or no call number from the host because the launch is being captured
+ * into a graph whose replays advance it): lane P loads call number and status from device memory, lane
+ * P + 1 the CTA count, whose top bit says that some CTA of this grid has already given up waiting; then
+ * the bounded wait.
+ *
+ * Returns the call number, or 0 with `give_up` telling why: 1 = not arrived within limit_ns, 2 = error
+ * or dead context.  `first` = the CTA's own tile (not a janitor's sweep).
+ */
+template <int P, int MODE>
+__device__ __forceinline__ uint32_t top_barrier(const ReduceArgs &a, size_t tile, unsigned long long limit_ns,
+                                                int &give_up, bool first)
 {
     __shared__ uint32_t s_epoch;
     __shared__ int s_why;
     DevState *st = a.st;
     __syncthreads();                                  /* the shared words may still be read from an earlier use */
     if (threadIdx.x < 32) {
-        const uint2 es = ld_relaxed_u32x2(&st->epoch);
-        const uint32_t e = entry_epoch(a, es);
-        int why = e ? 0 : 2;
-        int polls = 0;
-        if (e && threadIdx.x < P) {
-            polls = wait_flag_eq(&st->arrive[e & 1u][threadIdx.x], e, limit_ns);
-            if (polls < 0) { why = 1; polls = 0; }
+        const unsigned lane = threadIdx.x;
+        const uint32_t *fp = a.flags + (tile >> a.flag_shift) * kFlagStride + (lane < (unsigned)P ? lane : 0u);
+        uint32_t e = a.e_host, f = 0u;
+        int why = 0, polls = 0;
+        bool slow = (e == 0u);
+        if (!slow) {
+            if (lane < (unsigned)P) f = ld_acquire_u32(fp);
+            slow = !__all_sync(0xFFFFFFFFu, lane >= (unsigned)P || f == e);
         }
-        why = __reduce_max_sync(0xFFFFFFFFu, why);
-        polls = __reduce_add_sync(0xFFFFFFFFu, polls);
-        if (threadIdx.x == 0) {
+        if (slow) {
+            /* the relaxed loads first: an acquire load holds back what follows it in its thread */
+            uint2 es = make_uint2(0u, 0u);
+            uint32_t count = 0u;
+            if (lane == (unsigned)P) es = ld_relaxed_u32x2(&st->epoch);
+            if (lane == (unsigned)P + 1u) count = ld_relaxed_u32(&st->cta_arrive[a.parity]);
+            if (lane < (unsigned)P) f = ld_acquire_u32(fp);
+            es.x = __shfl_sync(0xFFFFFFFFu, es.x, P);
+            es.y = __shfl_sync(0xFFFFFFFFu, es.y, P);
+            count = __shfl_sync(0xFFFFFFFFu, count, P + 1);
+            if (first && predecessor_unpublished(a, es)) {
+                /* wait for the stream's previous kernel (this context's previous reducer), then look again */
+                gdc_wait();
+                if (lane == (unsigned)P) es = ld_relaxed_u32x2(&st->epoch);
+                es.x = __shfl_sync(0xFFFFFFFFu, es.x, P);
+                es.y = __shfl_sync(0xFFFFFFFFu, es.y, P);
+            }
+            e = entry_epoch(a, es);
+            why = e ? 0 : 2;
+            if (e && a.e_host && e != a.e_host) {     /* host and device disagree about the call number */
+                fail(st, a.host_status, SIFAR_ERR_EPOCH);
+                e = 0u; why = 2;
+            }
+            if (e) {
+                const bool ready = lane >= (unsigned)P || f == e;
+                if (!__all_sync(0xFFFFFFFFu, ready)) {
+                    if (first && a.two_phase && (count & kQueuedBit)) {
+                        why = 1;       /* the grid runs ahead of its producers: do not hold the SM, queue at once */
+                    } else if (!ready) {
+                        polls = wait_flag_eq(fp, e, limit_ns);
+                        if (polls < 0) { why = 1; polls = 0; }
+                        polls += 1;    /* the first look counts */
+                    }
+                }
+            }
+            why = __reduce_max_sync(0xFFFFFFFFu, why);
+            polls = __reduce_add_sync(0xFFFFFFFFu, polls);
+        }
+        if (lane == 0) {
             s_epoch = why ? 0u : e;
             s_why = why;
-            if (polls) atomicAdd(&st->stats[kStatFlagPolls], (unsigned long long)polls);
+            if (polls) {
+                atomicAdd(&st->stats[kStatFlagPolls], (unsigned long long)polls);
+                /* flagged tiles: a tile whose flags were not there at the first look is a mis-speculation */
+                if (MODE == kModeTiles && e) st_relaxed_u32(&st->retry_epoch, e);
+            }
         }
     }
     __syncthreads();
@@ -257,8 +350,6 @@ struct Roles {
     uint32_t ok;
 };
 
-constexpr uint32_t kQueuedBit = 0x80000000u;
-
 /* Thread 0 of a CTA in the deferring regime: queue the CTA's tile (made visible before the CTA's arrival). */
 __device__ __forceinline__ void defer_tile(const ReduceArgs &a, size_t tile)
 {
@@ -267,7 +358,7 @@ __device__ __forceinline__ void defer_tile(const ReduceArgs &a, size_t tile)
     __threadfence();
     /* "something is queued" travels in the top bit of the arrival count, set before this thread counts its
        CTA: who sees the count complete knows from the same word whether the queue needs a look */
-    asm volatile("red.relaxed.gpu.global.or.b32 [%0], %1;" :: "l"(&a.st->cta_arrive), "r"(kQueuedBit) : "memory");
+    asm volatile("red.relaxed.gpu.global.or.b32 [%0], %1;" :: "l"(&a.st->cta_arrive[a.parity]), "r"(kQueuedBit) : "memory");
 }
 
 /*
@@ -278,10 +369,15 @@ __device__ __forceinline__ void defer_tile(const ReduceArgs &a, size_t tile)
  *   Deferring: a CTA's SM slot is worth more than the answer, so it counts itself
  *   with a fire-and-forget increment and leaves.  The G CTAs with the highest
  *   indices (dispatched last) are the janitors: they wait until the count is
- *   complete and then learn how many tiles were queued.
- * A relaxed count is enough in both regimes: the CTA's loads have returned (its
- * stores depended on them), which is all the bottom barrier asks; `out` is handed
- * over by the kernel boundary; a queued tile was fenced by defer_tile().
+ *   complete and then learn from the same word whether anything was queued.
+ *   Nothing queued (the usual case): janitor 1 publishes, the others just leave.
+ * The count is polled with relaxed loads (half the round trip of an acquire); a
+ * fence follows only if the queue has to be read.  A relaxed count is enough in
+ * both regimes: the CTA's loads have returned (its stores depended on them),
+ * which is all the bottom barrier asks; `out` is handed over by the kernel
+ * boundary; a queued tile was fenced by defer_tile().  The word counts this
+ * call only (the other parity's word is re-armed by the CTA that publishes), so a
+ * janitor that looks late still finds it complete.
  */
 template <int MODE>
 __device__ __forceinline__ Roles cta_arrive(const ReduceArgs &a, uint32_t e, int P, bool alive, bool want_defer,
@@ -289,6 +385,7 @@ __device__ __forceinline__ Roles cta_arrive(const ReduceArgs &a, uint32_t e, int
 {
     __shared__ Roles s_roles;
     DevState *st = a.st;
+    uint32_t *counter = &st->cta_arrive[a.parity];
     const uint32_t n = gridDim.x;
     const bool janitor = a.two_phase && blockIdx.x + a.janitors >= n;
     /* One barrier: every thread's loads are done.  In place it also collects "somebody saw an error"; in
@@ -301,43 +398,31 @@ __device__ __forceinline__ Roles cta_arrive(const ReduceArgs &a, uint32_t e, int
         dead = __syncthreads_or(!alive);
     }
     if (a.two_phase && !janitor) {
-        if (!dead && threadIdx.x == 0) red_add_relaxed_u32(&st->cta_arrive, 1u);
+        if (!dead && threadIdx.x == 0) red_add_relaxed_u32(counter, 1u);
         return Roles{0u, 0u, (uint32_t)!dead};
     }
     if (threadIdx.x == 0) {
         Roles r = {0u, 0u, (uint32_t)!dead};
         if (!dead && !a.two_phase) {
-            const uint32_t arrived = (n > 1u) ? atom_add_relaxed_u32(&st->cta_arrive, 1u) + 1u : 1u;
-            if (arrived == n) {
-                if (n > 1u) st_relaxed_u32(&st->cta_arrive, 0u);
-                publish_call<MODE>(st, e, P);
-            }
+            const uint32_t arrived = (n > 1u) ? atom_add_relaxed_u32(counter, 1u) + 1u : 1u;
+            if (arrived == n) publish_call<MODE>(st, e, P);
         } else if (!dead) {
             r.janitor = blockIdx.x + a.janitors - n + 1u;              /* 1 .. G */
-            red_add_relaxed_u32(&st->cta_arrive, 1u);
-            /* Janitor 1 re-arms the counter as soon as it has seen it complete with nothing queued; a janitor
-               that polls a moment later would never see it complete.  So the wait also ends when the call
-               has been published, which in this phase only that fast path does. */
+            red_add_relaxed_u32(counter, 1u);
             Deadline d;
-            bool published = false, queued = false;
+            uint32_t count;
             for (;;) {
-                const uint2 es = ld_relaxed_u32x2(&st->epoch);         /* issued first: not held back by the acquire */
-                const uint32_t count = ld_acquire_u32(&st->cta_arrive); /* acquire: the queue entries of the CTAs counted */
-                queued = (count & kQueuedBit) != 0u;
+                count = ld_relaxed_u32(counter);
                 if ((count & ~kQueuedBit) >= n) break;
-                if (es.x == e) { published = true; break; }
-                if (es.y != 0u) { r.ok = 0u; break; }
                 if (d.expired(a.timeout_ns)) { fail(st, a.host_status, SIFAR_ERR_TIMEOUT); r.ok = 0u; break; }
+                if ((d.polls % 64u) == 0u && ld_relaxed_u32(&st->status) != 0u) { r.ok = 0u; break; }
             }
-            r.ndefer = (published || !queued) ? 0u : ld_relaxed_u32(a.defer);
-            if (published) {
-                r.janitor = 0u;
-            } else if (r.ok && r.ndefer == 0u) {
-                /* Nothing was queued (the usual case): janitor 1 publishes at once, the others just leave. */
-                if (r.janitor == 1u) {
-                    st_relaxed_u32(&st->cta_arrive, 0u);
-                    publish_call<MODE>(st, e, P);
-                }
+            if (r.ok && (count & kQueuedBit)) {
+                __threadfence();                                       /* the queue entries of the CTAs counted */
+                r.ndefer = ld_relaxed_u32(a.defer);
+            }
+            if (r.ok && r.ndefer == 0u) {
+                if (r.janitor == 1u) publish_call<MODE>(st, e, P);
                 r.janitor = 0u;
             }
         }
@@ -358,7 +443,7 @@ __device__ __forceinline__ void flush_reloads(DevState *st, uint32_t e, unsigned
     reloads = 0;
 }
 
-/* A janitor is done with its share (all threads call).  The last janitor re-arms the counters and publishes. */
+/* A janitor is done with its share (all threads call).  The last janitor re-arms the queue and publishes. */
 template <int MODE>
 __device__ __forceinline__ void janitor_leave(const ReduceArgs &a, uint32_t e, int P, bool alive)
 {
@@ -368,7 +453,6 @@ __device__ __forceinline__ void janitor_leave(const ReduceArgs &a, uint32_t e, i
         const uint32_t left = atom_add_relaxed_u32(&st->janitor_done, 1u) + 1u;
         if (left == a.janitors) {
             st_relaxed_u32(&st->janitor_done, 0u);
-            st_relaxed_u32(&st->cta_arrive, 0u);
             st_relaxed_u32(a.defer, 0u);
             publish_call<MODE>(st, e, P);
         }
@@ -382,14 +466,31 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a
     constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
     const size_t ntiles = tiles_for((size_t)a.n / EPV, U);
     const size_t tile = blockIdx.x;
-    /* programmatic dependent launch: nothing is read before the previous kernel of the stream is complete;
-       the next kernel may become resident as soon as every CTA of this one has started */
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;");
+    /* Programmatic dependent launch: the next kernel of the stream may become resident as soon as every
+       CTA of this one has started.  Whether this kernel's own reads wait for the kernel before it is the
+       host's choice (a.early, see launch_reduce); its writes always do. */
+    if (!a.early) gdc_wait();
+    gdc_launch_dependents();
     int give_up = 0;
-    uint32_t e = top_barrier<P>(a, a.two_phase ? a.spin_ns : a.timeout_ns, give_up);
+    if (a.early && (threadIdx.x & 7u) == 0u) {
+        /* While warp 0 makes its round trip for the flags, ask the L2 for the tile's lines (one thread per
+           128-byte line).  A prefetch returns nothing to the thread, so it cannot deliver stale data: the
+           loads below still follow the flags, and the L2 is where the producers' stores arrive. */
+        constexpr int EPVp = (DT == SIFAR_BF16) ? 8 : 4;
+        const size_t nvec = (size_t)a.n / EPVp;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t v = tile * kThreads * U + (size_t)u * kThreads + threadIdx.x;
+            if (v < nvec) {
+#pragma unroll
+                for (int r = 0; r < P; ++r) asm volatile("prefetch.global.L2 [%0];" :: "l"(a.src[r] + v));
+            }
+        }
+    }
+    uint32_t e = top_barrier<P, MODE>(a, tile, a.two_phase ? a.spin_ns : a.timeout_ns, give_up, true);
     bool alive = true;
     if (e == 0u) {
+        if (a.early) gdc_wait();                                       /* before anything is written */
         if (give_up == 2) return;                                      /* dead context */
         if (!a.two_phase) {
             if (threadIdx.x == 0) fail(a.st, a.host_status, SIFAR_ERR_TIMEOUT);
@@ -397,20 +498,23 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a
         }
         /* the ranks are late: queue the tile and free the SM; the call number is still needed to arrive */
         if (threadIdx.x == 0) defer_tile(a, tile);
-        e = entry_epoch(a, ld_relaxed_u32x2(&a.st->epoch));
+        e = entry_epoch(a, ld_relaxed_u32x2(&a.st->epoch));         /* after the wait: the predecessor has published */
         alive = (e != 0u);
     } else {
-        tile_plain<DT, P>(a, tile, ntiles);                            /* pull and reduce (phase 2) */
+        tile_plain<DT, P>(a, tile, ntiles, a.early != 0u);             /* pull and reduce (phase 2) */
     }
     /* phase 3 (bottom barrier, baseline only) and publication of the call number by the last CTA out */
     const Roles role = cta_arrive<MODE>(a, e, P, alive, false, tile);
     if (!role.janitor) return;
     alive = (role.ok != 0u);
-    if (alive && role.ndefer) {
-        alive = (top_barrier<P>(a, a.timeout_ns, give_up) != 0u);
-        if (!alive && give_up == 1 && threadIdx.x == 0) fail(a.st, a.host_status, SIFAR_ERR_TIMEOUT);
-        for (uint32_t i = role.janitor - 1u; i < role.ndefer && alive; i += a.janitors)
-            tile_plain<DT, P>(a, ld_relaxed_u32(a.defer + 1u + i), ntiles);
+    for (uint32_t i = role.janitor - 1u; i < role.ndefer && alive; i += a.janitors) {
+        const size_t t = ld_relaxed_u32(a.defer + 1u + i);
+        /* flagged tiles: the flags of each queued tile; barrier modes: the same P flags every time */
+        if (MODE == kModeTiles || i == role.janitor - 1u) {
+            alive = (top_barrier<P, MODE>(a, t, a.timeout_ns, give_up, false) != 0u);
+            if (!alive && give_up == 1 && threadIdx.x == 0) fail(a.st, a.host_status, SIFAR_ERR_TIMEOUT);
+        }
+        if (alive) tile_plain<DT, P>(a, t, ntiles, false);
     }
     janitor_leave<MODE>(a, e, P, alive);
 }
@@ -425,14 +529,15 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
     const size_t tile = blockIdx.x;
     const unsigned long long limit_ns = a.two_phase ? a.spin_ns : a.timeout_ns;
     unsigned reloads = 0;
-    /* programmatic dependent launch, as in k_reduce_plain */
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;");
+    /* programmatic dependent launch, as in k_reduce_plain: the slots validate themselves, so the loads
+       need not wait for the kernel before this one on the stream unless the host says so */
+    if (!a.early) gdc_wait();
+    gdc_launch_dependents();
 
     /* The call number is loaded together with the slots (no dependent round trip before the data), by one
        thread per CTA: a word that every warp of a large grid loads becomes a hot spot in its L2 slice. */
     __shared__ uint2 s_es;
-    if (threadIdx.x == 0) s_es = ld_relaxed_u32x2(&st->epoch);
+    if (threadIdx.x == 0) s_es = a.e_host ? make_uint2(a.e_host - 1u, 0u) : ld_relaxed_u32x2(&st->epoch);
     const size_t base = tile * kThreads * U + threadIdx.x;
     uint4 x[U][P];
 #pragma unroll
@@ -444,19 +549,35 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
         }
     }
     __syncthreads();
+    if (!a.e_host && predecessor_unpublished(a, s_es)) {    /* uniform over the CTA */
+        /* this context's previous reducer is still running ahead of us on the stream: wait for it and read
+           the call number again (what was loaded above is then stale and is loaded again by the validation) */
+        gdc_wait();
+        __syncthreads();
+        if (threadIdx.x == 0) s_es = ld_relaxed_u32x2(&st->epoch);
+        __syncthreads();
+    }
     const uint32_t e = entry_epoch(a, s_es);
     bool alive = (e != 0u);
     bool ok = true;
     if (alive) {
+        /* validation (Section 4.2): a slot counts iff it carries this call's tag; stale ones are re-loaded */
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const size_t s = base + (size_t)u * kThreads;
             if (s >= nslots || !ok) continue;
-            /* validation (Section 4.2): a slot counts iff it carries this call's tag; stale ones are re-loaded */
-            if (!validate_slot<P>(x[u], a.src, s, e, limit_ns, a.poll, reloads)) { ok = false; continue; }
-            store_slot_result<DT>(a.out, s, (size_t)a.n, sum_vec<DT, P>(x[u], false));
+            ok = validate_slot<P>(x[u], a.src, s, e, limit_ns, a.poll, reloads);
         }
-        if (!a.two_phase && !ok) {
+    }
+    if (a.early) gdc_wait();                                /* everything from here on writes */
+    if (alive) {
+        if (ok) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const size_t s = base + (size_t)u * kThreads;
+                if (s < nslots) store_slot_result<DT>(a.out, s, (size_t)a.n, sum_vec<DT, P>(x[u], false));
+            }
+        } else if (!a.two_phase) {
             fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
             alive = false;
         }
@@ -492,7 +613,10 @@ __device__ __forceinline__ void pack_body(const PackArgs &a)
         const uint2 es = ld_relaxed_u32x2(&st->epoch);
         uint32_t e = es.x + 1u;
         bool ok = (es.y == 0u);
-        if (ok && MODE != SIFAR_BARRIER_ONESHOT && (e & 1u) != a.parity) {
+        /* The call number is the device's, so this producer must be ordered after the previous call's reducer
+           (stream, event or graph edge).  One that was not reads a call number that is one short: its parity
+           differs from what the host enqueued it for. */
+        if (ok && (e & 1u) != a.parity) {
             fail(st, a.host_status, SIFAR_ERR_EPOCH);
             ok = false;
         }
@@ -511,7 +635,38 @@ __device__ __forceinline__ void pack_body(const PackArgs &a)
 
     const size_t tid = (size_t)blockIdx.x * kThreads + threadIdx.x;
     const size_t nthreads = (size_t)gridDim.x * kThreads;
-    if (MODE != SIFAR_SPECULATIVE) {
+    if (MODE == kModeTiles) {
+        /* Flagged tiles: plain data, and one arrival flag per block of kFlagBlockVecs vectors, released as soon
+           as the block is stored, so that the reducer can start on it while the rest is still being written.
+           One block per CTA and round, four vectors per thread in flight.  The releasing thread changes from
+           round to round: its fence then overlaps the next round's loads of the other warps. */
+        constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
+        constexpr int VPT = (int)(kFlagBlockVecs / kThreads);
+        const size_t nvec = (size_t)a.n / EPV;
+        const size_t nblocks = nvec ? (nvec + kFlagBlockVecs - 1) / kFlagBlockVecs : 1;
+        const uint4 *src = reinterpret_cast<const uint4 *>(a.src);
+        uint4 *dst = reinterpret_cast<uint4 *>(a.dst);
+        unsigned round = 0;
+        for (size_t b = blockIdx.x; b < nblocks; b += gridDim.x, ++round) {
+            const size_t v0 = b * kFlagBlockVecs + threadIdx.x;
+            uint4 x[VPT];
+#pragma unroll
+            for (int j = 0; j < VPT; ++j)
+                if (v0 + (size_t)j * kThreads < nvec) x[j] = __ldcs(src + v0 + (size_t)j * kThreads);
+#pragma unroll
+            for (int j = 0; j < VPT; ++j)
+                if (v0 + (size_t)j * kThreads < nvec) st_slot(dst + v0 + (size_t)j * kThreads, x[j]);
+            const size_t i = nvec * EPV + threadIdx.x;                 /* ragged tail, with the last block */
+            if (b == nblocks - 1 && i < a.n) {
+                if (DT == SIFAR_BF16)
+                    reinterpret_cast<uint16_t *>(a.dst)[i] = reinterpret_cast<const uint16_t *>(a.src)[i];
+                else
+                    reinterpret_cast<uint32_t *>(a.dst)[i] = reinterpret_cast<const uint32_t *>(a.src)[i];
+            }
+            __syncthreads();
+            if (threadIdx.x == ((round * 32u) % kThreads)) st_release_u32(a.tile_flags + b * kFlagStride + a.rank, e);
+        }
+    } else if (MODE != SIFAR_SPECULATIVE) {
         constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
         const size_t nvec = (size_t)a.n / EPV;
         const uint4 *src = reinterpret_cast<const uint4 *>(a.src);
@@ -593,22 +748,24 @@ __global__ void __launch_bounds__(kThreads) k_pack_all(const PackAllArgs all)
 }
 
 /* Release of one rank's arrival flag after caller-written plain partials. */
-__global__ void k_arrive(DevState *st, uint32_t rank)
+__global__ void k_arrive(DevState *st, int *host_status, uint32_t rank, uint32_t parity)
 {
     const uint2 es = ld_relaxed_u32x2(&st->epoch);
     if (es.y != 0u) return;
     const uint32_t e = es.x + 1u;
+    if ((e & 1u) != parity) { fail(st, host_status, SIFAR_ERR_EPOCH); return; }   /* not ordered after the previous call */
     __threadfence();
     st_release_u32(&st->arrive[e & 1u][rank], e);
 }
 
 /* Producer-side half of the bottom barrier as a kernel of its own. */
-__global__ void k_wait_writable(DevState *st, int *host_status, uint32_t rank, uint32_t wait_delta,
+__global__ void k_wait_writable(DevState *st, int *host_status, uint32_t rank, uint32_t wait_delta, uint32_t parity,
                                 unsigned long long timeout_ns)
 {
     const uint2 es = ld_relaxed_u32x2(&st->epoch);
     if (es.y != 0u) return;
     const uint32_t e = es.x + 1u;
+    if ((e & 1u) != parity) { fail(st, host_status, SIFAR_ERR_EPOCH); return; }
     if (wait_flag_ge(&st->done[rank], e - wait_delta, timeout_ns) < 0) fail(st, host_status, SIFAR_ERR_TIMEOUT);
 }
 
@@ -619,6 +776,7 @@ __global__ void k_empty_call(DevState *st, int mode, int P)
     if (es.y != 0u) return;
     const uint32_t e = es.x + 1u;
     st->stats[kStatCalls] += 1ull;
+    st->cta_arrive[(e + 1u) & 1u] = 0u;             /* what the CTA that closes a call does for the next one */
     if (mode == SIFAR_BARRIER_ONESHOT) {
         __threadfence();
         for (int r = 0; r < P; ++r) st_relaxed_u32(&st->done[r], e);
@@ -626,7 +784,7 @@ __global__ void k_empty_call(DevState *st, int mode, int P)
     st_release_u32(&st->epoch, e);
 }
 
-__global__ void k_set_epoch(DevState *st, uint32_t e) { st->epoch = e; }
+__global__ void k_set_epoch(DevState *st, uint32_t e) { st->epoch = e; st->cta_arrive[0] = 0u; st->cta_arrive[1] = 0u; }
 
 /* ------------------------------------------------------------------------ */
 /* launch geometry                                                           */
@@ -674,6 +832,7 @@ static cudaError_t launch_reduce_p(int mode, int grid, cudaStream_t s, const Red
     switch (mode) {
     case SIFAR_BARRIER_ONESHOT: return launch_k(k_reduce_plain<DT, P, SIFAR_BARRIER_ONESHOT>, grid, s, a);
     case SIFAR_DUALBUF:         return launch_k(k_reduce_plain<DT, P, SIFAR_DUALBUF>, grid, s, a);
+    case kModeTiles:            return launch_k(k_reduce_plain<DT, P, kModeTiles>, grid, s, a);
     default:                    return launch_k(k_reduce_spec<DT, P>, grid, s, a);
     }
 }
@@ -709,18 +868,35 @@ sifar::PollShape sifar::poll_shape_for(const sifar_ctx *ctx, size_t n)
 
 static int unroll_for(int P) { return P <= 2 ? 4 : P <= 4 ? 2 : 1; }
 
-static size_t reduce_units(const sifar_ctx *ctx, size_t n, int mode)
+/* 16-byte units the reducer works on: slots, or vectors of plain elements (kernel mode, see kModeTiles). */
+static size_t reduce_units(const sifar_ctx *ctx, size_t n, int kernel_mode)
 {
-    return mode == SIFAR_SPECULATIVE ? sifar::slots_for(ctx->dtype, n) : n * sifar::elem_size(ctx->dtype) / 16;
+    return kernel_mode == SIFAR_SPECULATIVE ? sifar::slots_for(ctx->dtype, n)
+                                            : n * sifar::elem_size(ctx->dtype) / 16;
 }
 
+/* The chains use the slot format at every size. */
 size_t sifar::reduce_tiles(const sifar_ctx *ctx, size_t n, int mode)
 {
     return tiles_for(reduce_units(ctx, n, mode), unroll_for(ctx->P));
 }
 
-/* Kernels one all-reduce call launches. */
-int sifar::reduce_launch_count(const sifar_ctx *, size_t, int) { return 1; }
+/*
+ * Format of the speculative mode by size.  Slots carry their own tags (no flag, no dependent round trip)
+ * but move a third more bytes; from 16 MiB for all P partials together, where bandwidth is what counts,
+ * the partial travels as plain data with one arrival flag per 16 KiB block.
+ */
+static int spec_format(int P, int dtype, size_t n)
+{
+    constexpr size_t kTilesFromBytes = (size_t)16 << 20;
+    return (size_t)P * n * sifar::elem_size(dtype) < kTilesFromBytes ? SIFAR_FORMAT_SLOTS : SIFAR_FORMAT_TILES;
+}
+
+static size_t flag_blocks(int dtype, size_t n)
+{
+    const size_t nvec = n * sifar::elem_size(dtype) / 16;
+    return nvec ? (nvec + sifar::kFlagBlockVecs - 1) / sifar::kFlagBlockVecs : 1;
+}
 
 namespace sifar {
 
@@ -731,6 +907,7 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
         SIFAR_CUDA(cudaGetLastError());
         return SIFAR_OK;
     }
+    const int kernel_mode = (rl.mode == SIFAR_SPECULATIVE && rl.format == SIFAR_FORMAT_TILES) ? kModeTiles : rl.mode;
     ReduceArgs a;
     memset(&a, 0, sizeof a);
     for (int r = 0; r < ctx->P; ++r) a.src[r] = reinterpret_cast<const uint4 *>(rl.src[r]);
@@ -740,22 +917,101 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
     a.host_status = ctx->d_status_alias;
     a.timeout_ns = ctx->timeout_ns;
     a.parity = rl.parity;
-    a.check_parity = (rl.mode != SIFAR_BARRIER_ONESHOT);
+    a.check_parity = 1u;
     a.poll = poll_shape_for(ctx, rl.n);
     a.defer = ctx->d_defer;
     a.spin_ns = ctx->spin_ns < ctx->timeout_ns ? ctx->spin_ns : ctx->timeout_ns;
     /* One tile per CTA.  Up to one CTA per SM the reducer cannot crowd out the producers and waits in
-       place; beyond that it runs at full occupancy, waits briefly, and its last CTAs sweep up. */
-    const size_t ntiles = tiles_for(reduce_units(ctx, rl.n, rl.mode), unroll_for(ctx->P));
+       place; beyond that it runs at full occupancy, waits briefly, and its last CTAs sweep up.  Two
+       janitors per SM: half the registers of an SM stay free for the producers they wait for, and the
+       sweep still runs at three quarters of the full-occupancy bandwidth. */
+    const int U = unroll_for(ctx->P);
+    const size_t ntiles = tiles_for(reduce_units(ctx, rl.n, kernel_mode), U);
     a.two_phase = ntiles > (size_t)ctx->sm_count ? 1u : 0u;
-    a.janitors = (uint32_t)ctx->sm_count;
+    a.janitors = (uint32_t)ctx->sm_count * 2u;
+    if (a.janitors > ntiles) a.janitors = (uint32_t)ntiles;
+    if (kernel_mode == kModeTiles) {
+        /* a tile is kThreads * U vectors, a flag block kFlagBlockVecs = 4 * kThreads vectors */
+        a.flags = rl.tile_flags;
+        a.flag_shift = U == 1 ? 2u : U == 2 ? 1u : 0u;
+    } else {
+        a.flags = &ctx->d_state->arrive[rl.parity][0];
+        a.flag_shift = 31u;
+    }
+    /* The call number: the host's own count, unless this launch is being captured into a graph, whose
+       replays advance the number in device memory. */
+    a.e_host = 0u;
+    if (rl.e_host) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusActive;
+        if (cudaStreamIsCapturing(stream, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone) a.e_host = rl.e_host;
+        else cudaGetLastError();
+    }
+    /* Early reads need programmatic launch to mean anything, and the baseline keeps the plain stream order. */
+    a.early = (rl.early && g_pdl && a.two_phase && rl.mode != SIFAR_BARRIER_ONESHOT && !rl.programmatic_event) ? 1u : 0u;
     g_programmatic_event = rl.programmatic_event;
     cudaError_t err = (ctx->dtype == SIFAR_BF16)
-        ? launch_reduce_dt<SIFAR_BF16>(ctx->P, rl.mode, (int)ntiles, stream, a)
-        : launch_reduce_dt<SIFAR_F32>(ctx->P, rl.mode, (int)ntiles, stream, a);
+        ? launch_reduce_dt<SIFAR_BF16>(ctx->P, kernel_mode, (int)ntiles, stream, a)
+        : launch_reduce_dt<SIFAR_F32>(ctx->P, kernel_mode, (int)ntiles, stream, a);
     g_programmatic_event = nullptr;
     SIFAR_CUDA(err);
     return SIFAR_OK;
+}
+
+/*
+ * With lazy module loading (the CUDA default) the first launch of a kernel loads its code, and that load
+ * can wait for the device to become idle.  Producers are routinely launched for the first time while a
+ * reducer is already polling for them, so such a launch would block on the host until the reducer gave
+ * up.  Every kernel of a context's shape is therefore loaded when the context is created.
+ */
+template <typename K>
+static cudaError_t preload(K kernel)
+{
+    cudaFuncAttributes at;
+    return cudaFuncGetAttributes(&at, kernel);
+}
+
+template <int DT, int P>
+static cudaError_t preload_reducers()
+{
+    cudaError_t e = preload(k_reduce_plain<DT, P, SIFAR_BARRIER_ONESHOT>);
+    if (e == cudaSuccess) e = preload(k_reduce_plain<DT, P, SIFAR_DUALBUF>);
+    if (e == cudaSuccess) e = preload(k_reduce_plain<DT, P, kModeTiles>);
+    if (e == cudaSuccess) e = preload(k_reduce_spec<DT, P>);
+    return e;
+}
+
+template <int DT>
+static cudaError_t preload_dt(int P)
+{
+    cudaError_t e = cudaSuccess;
+    switch (P) {
+    case 1: e = preload_reducers<DT, 1>(); break;
+    case 2: e = preload_reducers<DT, 2>(); break;
+    case 3: e = preload_reducers<DT, 3>(); break;
+    case 4: e = preload_reducers<DT, 4>(); break;
+    case 5: e = preload_reducers<DT, 5>(); break;
+    case 6: e = preload_reducers<DT, 6>(); break;
+    case 7: e = preload_reducers<DT, 7>(); break;
+    default: e = preload_reducers<DT, 8>(); break;
+    }
+    if (e == cudaSuccess) e = preload(k_pack<DT, SIFAR_BARRIER_ONESHOT>);
+    if (e == cudaSuccess) e = preload(k_pack<DT, SIFAR_DUALBUF>);
+    if (e == cudaSuccess) e = preload(k_pack<DT, SIFAR_SPECULATIVE>);
+    if (e == cudaSuccess) e = preload(k_pack<DT, kModeTiles>);
+    if (e == cudaSuccess) e = preload(k_pack_all<DT, SIFAR_BARRIER_ONESHOT>);
+    if (e == cudaSuccess) e = preload(k_pack_all<DT, SIFAR_DUALBUF>);
+    if (e == cudaSuccess) e = preload(k_pack_all<DT, SIFAR_SPECULATIVE>);
+    if (e == cudaSuccess) e = preload(k_pack_all<DT, kModeTiles>);
+    if (e == cudaSuccess) e = preload(k_arrive);
+    if (e == cudaSuccess) e = preload(k_wait_writable);
+    if (e == cudaSuccess) e = preload(k_empty_call);
+    if (e == cudaSuccess) e = preload(k_set_epoch);
+    return e;
+}
+
+cudaError_t preload_kernels(int dtype, int P)
+{
+    return dtype == SIFAR_BF16 ? preload_dt<SIFAR_BF16>(P) : preload_dt<SIFAR_F32>(P);
 }
 
 template <int DT>
@@ -764,6 +1020,7 @@ static cudaError_t launch_pack_all_dt(int mode, dim3 grid, cudaStream_t s, const
     switch (mode) {
     case SIFAR_BARRIER_ONESHOT: k_pack_all<DT, SIFAR_BARRIER_ONESHOT><<<grid, kThreads, 0, s>>>(a); break;
     case SIFAR_DUALBUF:         k_pack_all<DT, SIFAR_DUALBUF><<<grid, kThreads, 0, s>>>(a); break;
+    case kModeTiles:            k_pack_all<DT, kModeTiles><<<grid, kThreads, 0, s>>>(a); break;
     default:                    k_pack_all<DT, SIFAR_SPECULATIVE><<<grid, kThreads, 0, s>>>(a); break;
     }
     return cudaGetLastError();
@@ -775,6 +1032,7 @@ static cudaError_t launch_pack_dt(int mode, int grid, cudaStream_t s, const Pack
     switch (mode) {
     case SIFAR_BARRIER_ONESHOT: k_pack<DT, SIFAR_BARRIER_ONESHOT><<<grid, kThreads, 0, s>>>(a); break;
     case SIFAR_DUALBUF:         k_pack<DT, SIFAR_DUALBUF><<<grid, kThreads, 0, s>>>(a); break;
+    case kModeTiles:            k_pack<DT, kModeTiles><<<grid, kThreads, 0, s>>>(a); break;
     default:                    k_pack<DT, SIFAR_SPECULATIVE><<<grid, kThreads, 0, s>>>(a); break;
     }
     return cudaGetLastError();
@@ -802,21 +1060,22 @@ extern "C" size_t sifar_algorithmic_bytes(int P, int dtype, size_t n, int mode)
 {
     if (!valid_dtype(dtype) || !valid_mode(mode) || P < 1) return 0;
     const size_t payload = n * elem_size(dtype);
-    const size_t per_rank = (mode == SIFAR_SPECULATIVE) ? slots_for(dtype, n) * 16 : payload;
+    const bool slots = (mode == SIFAR_SPECULATIVE && spec_format(P, dtype, n) == SIFAR_FORMAT_SLOTS);
+    const size_t per_rank = slots ? slots_for(dtype, n) * 16 : payload;
     size_t flags = 0;
+    if (mode == SIFAR_SPECULATIVE && !slots) flags += (size_t)P * 4 * flag_blocks(dtype, n);   /* one flag per block */
     if (mode != SIFAR_SPECULATIVE) flags += (size_t)P * 4;          /* arrival flags */
     if (mode == SIFAR_BARRIER_ONESHOT) flags += (size_t)P * 4;      /* done flags    */
     return (size_t)P * per_rank + payload + flags;
 }
 
-extern "C" int sifar_mode_for_payload(int P, int dtype, size_t n)
+extern "C" int sifar_spec_format(int P, int dtype, size_t n)
 {
     if (P < 1 || P > kMaxRanks || !valid_dtype(dtype)) {
-        set_error("sifar_mode_for_payload: need 1 <= P <= %d and a known dtype", kMaxRanks);
+        set_error("sifar_spec_format: need 1 <= P <= %d and a known dtype", kMaxRanks);
         return SIFAR_ERR_INVALID;
     }
-    constexpr size_t kSpeculativeBelowBytes = (size_t)16 << 20;     /* all P partials together */
-    return (size_t)P * n * elem_size(dtype) < kSpeculativeBelowBytes ? SIFAR_SPECULATIVE : SIFAR_DUALBUF;
+    return spec_format(P, dtype, n);
 }
 
 extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
@@ -857,12 +1116,18 @@ extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
     const size_t defer_words = 2 + (slots_for(dtype, max_elems) + kThreads - 1) / kThreads;
     if (e == cudaSuccess) e = cudaMalloc(&c->d_defer, defer_words * sizeof(uint32_t));
     if (e == cudaSuccess) e = cudaMemset(c->d_defer, 0, defer_words * sizeof(uint32_t));
+    /* arrival flags of the flagged-tile format: one word per block, rank and parity; 0 = never valid */
+    c->tflag_words = round_up((flag_blocks(dtype, max_elems) + 1) * kFlagStride, 32);
+    const size_t tflag_bytes = c->tflag_words * 2 * sizeof(uint32_t);
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_tflags, tflag_bytes);
+    if (e == cudaSuccess) e = cudaMemset(c->d_tflags, 0, tflag_bytes);
     if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->h_status, sizeof(int), cudaHostAllocMapped);
     if (e == cudaSuccess) { *c->h_status = 0; e = cudaHostGetDevicePointer((void **)&c->d_status_alias, (void *)c->h_status, 0); }
     if (e == cudaSuccess) e = cudaMemset(c->d_plain, 0, plain_bytes);
     if (e == cudaSuccess) e = cudaMemset(c->d_slots, 0, slot_bytes);
     if (e == cudaSuccess) e = cudaMemset(c->d_state, 0, sizeof(DevState));
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->host_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = preload_kernels(dtype, P);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         set_error("sifar_create: %s", cudaGetErrorString(e));
@@ -872,6 +1137,7 @@ extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
         if (c->d_slots) cudaFree(c->d_slots);
         if (c->d_state) cudaFree(c->d_state);
         if (c->d_defer) cudaFree(c->d_defer);
+        if (c->d_tflags) cudaFree(c->d_tflags);
         if (c->h_status) cudaFreeHost((void *)c->h_status);
         if (c->host_stream) cudaStreamDestroy(c->host_stream);
         delete c;
@@ -890,6 +1156,7 @@ extern "C" int sifar_destroy(sifar_ctx *c)
     cudaFree(c->d_slots);
     cudaFree(c->d_state);
     cudaFree(c->d_defer);
+    cudaFree(c->d_tflags);
     if (c->d_stage_in) cudaFree(c->d_stage_in);
     if (c->d_stage_out) cudaFree(c->d_stage_out);
     cudaFreeHost((void *)c->h_status);
@@ -926,7 +1193,16 @@ static const void *ctx_buffer(const sifar_ctx *c, int mode, uint32_t e, int r)
 
 static size_t ctx_buffer_bytes(const sifar_ctx *c, int mode, size_t n)
 {
-    return mode == SIFAR_SPECULATIVE ? slots_for(c->dtype, n) * 16 : n * elem_size(c->dtype);
+    const bool slots = (mode == SIFAR_SPECULATIVE && spec_format(c->P, c->dtype, n) == SIFAR_FORMAT_SLOTS);
+    return slots ? slots_for(c->dtype, n) * 16 : n * elem_size(c->dtype);
+}
+
+/* What sifar_pack / sifar_arrive remember about the producer of `rank` for call e. */
+static void note_producer(sifar_ctx *c, int rank, uint32_t e, cudaStream_t stream, size_t n)
+{
+    c->prod_epoch[rank] = e;
+    c->prod_stream[rank] = stream;
+    c->prod_n[rank] = n;
 }
 
 static bool overlaps(const void *a, size_t na, const void *b, size_t nb)
@@ -972,7 +1248,24 @@ extern "C" int sifar_allreduce(sifar_ctx *c, const void *const *rank_ptrs, void 
         }
         rl.src[r] = p;
     }
-    rl.out = out; rl.n = n; rl.mode = mode; rl.parity = e & 1u;
+    rl.out = out; rl.n = n; rl.mode = mode; rl.parity = e & 1u; rl.e_host = e;
+    rl.format = (mode == SIFAR_SPECULATIVE) ? spec_format(c->P, c->dtype, n) : SIFAR_FORMAT_SLOTS;
+    /* Where every rank's producer of this call is known to have been enqueued on another stream, nothing
+       this reducer reads is produced by the kernel before it on its own stream, and its loads may start
+       while that kernel drains (its writes still wait).  Unknown producers (partials stored by the
+       caller's own kernels without sifar_arrive) or the same stream: the plain stream order. */
+    rl.early = (stream != nullptr);
+    for (int r = 0; r < c->P; ++r) {
+        if (c->prod_epoch[r] != e) { rl.early = false; continue; }
+        if (c->prod_stream[r] == (cudaStream_t)stream || c->prod_stream[r] == nullptr) rl.early = false;
+        if (c->prod_n[r] != (size_t)-1 && c->prod_n[r] != n && mode == SIFAR_SPECULATIVE &&
+            spec_format(c->P, c->dtype, c->prod_n[r]) != rl.format) {
+            set_error("sifar_allreduce: rank %d was packed for %zu elements, whose speculative format differs "
+                      "from that of n = %zu", r, c->prod_n[r], n);
+            return SIFAR_ERR_INVALID;
+        }
+    }
+    rl.tile_flags = c->tile_flags((int)(e & 1u));
     rc = launch_reduce(c, rl, (cudaStream_t)stream);
     if (rc) return rc;
     c->h_epoch = e;
@@ -992,6 +1285,18 @@ extern "C" int sifar_rank_buffer(sifar_ctx *c, int rank, int mode, void **ptr, u
     if (rc) return rc;
     if (ptr) *ptr = const_cast<void *>(ctx_buffer(c, mode, e, rank));
     if (epoch) *epoch = e;
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_tile_flags(sifar_ctx *c, int rank, void **flags, size_t *elems_per_flag, size_t *stride_words)
+{
+    if (!c || rank < 0 || rank >= c->P) { set_error("sifar_tile_flags: NULL context or bad rank"); return SIFAR_ERR_INVALID; }
+    uint32_t e;
+    int rc = next_epoch(c, "sifar_tile_flags", &e);
+    if (rc) return rc;
+    if (flags) *flags = c->tile_flags((int)(e & 1u)) + rank;
+    if (elems_per_flag) *elems_per_flag = kFlagBlockVecs * 16 / elem_size(c->dtype);
+    if (stride_words) *stride_words = kFlagStride;
     return SIFAR_OK;
 }
 
@@ -1020,16 +1325,22 @@ extern "C" int sifar_pack(sifar_ctx *c, int rank, const void *src, size_t n, int
     a.rank = (uint32_t)rank;
     a.parity = e & 1u;
     a.wait_delta = (mode == SIFAR_BARRIER_ONESHOT && c->last_mode0_epoch) ? e - c->last_mode0_epoch : 0u;
-    const size_t units = (mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, n) : (n * elem_size(c->dtype) + 15) / 16;
-    size_t grid = (units + kThreads - 1) / kThreads;
+    a.tile_flags = c->tile_flags((int)(e & 1u));
+    const int kernel_mode = (mode == SIFAR_SPECULATIVE && spec_format(c->P, c->dtype, n) == SIFAR_FORMAT_TILES)
+                                ? kModeTiles : mode;
+    const size_t units = (kernel_mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, n)
+                                                            : (n * elem_size(c->dtype) + 15) / 16;
+    size_t grid = (kernel_mode == kModeTiles) ? flag_blocks(c->dtype, n) : (units + kThreads - 1) / kThreads;
     /* two CTAs per SM: the P ranks pack at the same time on their own streams (measured: 5.4-5.5 TB/s for eight
        ranks together; four or eight CTAs per SM were slower together and little faster alone) */
     const size_t cap = (size_t)c->sm_count * 2;
     if (grid > cap) grid = cap;
     if (grid < 1) grid = 1;
-    cudaError_t err = (c->dtype == SIFAR_BF16) ? launch_pack_dt<SIFAR_BF16>(mode, (int)grid, (cudaStream_t)stream, a)
-                                               : launch_pack_dt<SIFAR_F32>(mode, (int)grid, (cudaStream_t)stream, a);
+    cudaError_t err = (c->dtype == SIFAR_BF16)
+        ? launch_pack_dt<SIFAR_BF16>(kernel_mode, (int)grid, (cudaStream_t)stream, a)
+        : launch_pack_dt<SIFAR_F32>(kernel_mode, (int)grid, (cudaStream_t)stream, a);
     SIFAR_CUDA(err);
+    note_producer(c, rank, e, (cudaStream_t)stream, n);
     return SIFAR_OK;
 }
 
@@ -1041,8 +1352,11 @@ extern "C" int sifar_arrive(sifar_ctx *c, int rank, int mode, void *stream)
         set_error("sifar_arrive: bad rank, or a mode without arrival flags");
         return SIFAR_ERR_INVALID;
     }
-    k_arrive<<<1, 1, 0, (cudaStream_t)stream>>>(c->d_state, (uint32_t)rank);
+    uint32_t e;
+    if ((rc = next_epoch(c, "sifar_arrive", &e))) return rc;
+    k_arrive<<<1, 1, 0, (cudaStream_t)stream>>>(c->d_state, c->d_status_alias, (uint32_t)rank, e & 1u);
     SIFAR_CUDA(cudaGetLastError());
+    note_producer(c, rank, e, (cudaStream_t)stream, (size_t)-1);
     return SIFAR_OK;
 }
 
@@ -1054,7 +1368,7 @@ extern "C" int sifar_wait_writable(sifar_ctx *c, int rank, void *stream)
     if (!c->last_mode0_epoch) return SIFAR_OK;      /* nothing has read the buffer yet */
     const uint32_t delta = c->h_epoch + 1u - c->last_mode0_epoch;
     k_wait_writable<<<1, 1, 0, (cudaStream_t)stream>>>(c->d_state, c->d_status_alias, (uint32_t)rank, delta,
-                                                       c->timeout_ns);
+                                                       (c->h_epoch + 1u) & 1u, c->timeout_ns);
     SIFAR_CUDA(cudaGetLastError());
     return SIFAR_OK;
 }
@@ -1091,10 +1405,12 @@ extern "C" int sifar_reset(sifar_ctx *c, void *stream)
     SIFAR_CUDA(cudaMemsetAsync(c->d_slots, 0, c->slot_stride * 2 * c->P, s));
     SIFAR_CUDA(cudaMemsetAsync(c->d_state, 0, sizeof(DevState), s));
     SIFAR_CUDA(cudaMemsetAsync(c->d_defer, 0, sizeof(uint32_t), s));
+    SIFAR_CUDA(cudaMemsetAsync(c->d_tflags, 0, c->tflag_words * 2 * sizeof(uint32_t), s));
     SIFAR_CUDA(cudaStreamSynchronize(s));
     *c->h_status = 0;
     c->h_epoch = 0;
     c->last_mode0_epoch = 0;
+    memset(c->prod_epoch, 0, sizeof c->prod_epoch);
     return SIFAR_OK;
 }
 
@@ -1107,6 +1423,7 @@ extern "C" int sifar_debug_set_epoch(sifar_ctx *c, unsigned calls_so_far)
     SIFAR_CUDA(cudaDeviceSynchronize());
     c->h_epoch = calls_so_far;
     c->last_mode0_epoch = 0;
+    memset(c->prod_epoch, 0, sizeof c->prod_epoch);
     return SIFAR_OK;
 }
 
@@ -1156,20 +1473,24 @@ extern "C" int sifar_allreduce_host(sifar_ctx *c, const void *const *host_rank_p
         uint32_t e;
         if ((rc = next_epoch(c, "sifar_allreduce_host", &e))) return rc;
         for (int r = 0; r < c->P; ++r) all.dst[r] = const_cast<void *>(ctx_buffer(c, mode, e, r));
+        all.common.tile_flags = c->tile_flags((int)(e & 1u));
+        const int kernel_mode = (mode == SIFAR_SPECULATIVE && spec_format(c->P, c->dtype, n) == SIFAR_FORMAT_TILES)
+                                    ? kModeTiles : mode;
         all.common.n = n;
         all.common.st = c->d_state;
         all.common.host_status = c->d_status_alias;
         all.common.timeout_ns = c->timeout_ns;
         all.common.parity = e & 1u;
         all.common.wait_delta = (mode == SIFAR_BARRIER_ONESHOT && c->last_mode0_epoch) ? e - c->last_mode0_epoch : 0u;
-        const size_t units = (mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, n) : (bytes + 15) / 16;
-        size_t gx = (units + kThreads - 1) / kThreads;
+        const size_t units = (kernel_mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, n) : (bytes + 15) / 16;
+        size_t gx = (kernel_mode == kModeTiles) ? flag_blocks(c->dtype, n) : (units + kThreads - 1) / kThreads;
         const size_t cap = (size_t)c->sm_count * 2;
         if (gx > cap) gx = cap;
         cudaError_t err = (c->dtype == SIFAR_BF16)
-            ? launch_pack_all_dt<SIFAR_BF16>(mode, dim3((unsigned)gx, (unsigned)c->P), s, all)
-            : launch_pack_all_dt<SIFAR_F32>(mode, dim3((unsigned)gx, (unsigned)c->P), s, all);
+            ? launch_pack_all_dt<SIFAR_BF16>(kernel_mode, dim3((unsigned)gx, (unsigned)c->P), s, all)
+            : launch_pack_all_dt<SIFAR_F32>(kernel_mode, dim3((unsigned)gx, (unsigned)c->P), s, all);
         SIFAR_CUDA(err);
+        for (int r = 0; r < c->P; ++r) note_producer(c, r, e, s, n);
         void *out_dev = device_view(host_out);
         if (out_dev && ((uintptr_t)out_dev & 15u) == 0) {
             if ((rc = sifar_allreduce(c, nullptr, out_dev, n, mode, s))) return rc;     /* result written in place */

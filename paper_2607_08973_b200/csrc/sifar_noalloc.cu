@@ -140,6 +140,19 @@ using namespace sifar;
 
 extern "C" size_t sifar_noalloc_max_elems(void) { return kNoallocMaxElems; }
 
+extern "C" int sifar_noalloc_counters(unsigned long long out[3])
+{
+    if (!out) { set_error("sifar_noalloc_counters: NULL destination"); return SIFAR_ERR_INVALID; }
+    NoallocScratch *scratch = nullptr;
+    int rc = noalloc_scratch(&scratch);
+    if (rc) return rc;
+    NoallocScratch h;
+    SIFAR_CUDA(cudaDeviceSynchronize());
+    SIFAR_CUDA(cudaMemcpy(&h, scratch, sizeof h, cudaMemcpyDeviceToHost));    /* to a host stack object: no allocation */
+    out[0] = h.cta_arrive; out[1] = h.calls; out[2] = h.elements;
+    return SIFAR_OK;
+}
+
 extern "C" int sifar_allreduce_noalloc(const void *const *rank_ptrs, int P, void *out, size_t n, int dtype,
                                        void *stream)
 {

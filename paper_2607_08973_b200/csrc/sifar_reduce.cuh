@@ -215,7 +215,7 @@ __device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const 
 {
     if (!validate_once<P>(x, src, s, e, timeout_ns, shape, reloads, round_stamps)) return false;
     if (shape.forced == 0u) return true;
-    /* Forced retries (the retry-latency experiment of Section 7, "Retry Overhead"): the attempt that found
+    /* Forced retries (the retry-latency experiment of Section 6.3, "Retry Overhead"): the attempt that found
        every copy valid is treated as mis-speculated, `forced` times: each round loads all P copies again.
        The address of a round depends on the previous round's tags through a zero the compiler cannot see,
        so the rounds run one after another as real retries do.  The last copies are validated as usual

@@ -164,6 +164,46 @@ __global__ void k_delays(sifar_workload w, int P, uint32_t t, unsigned *out)
 
 __global__ void k_spin(unsigned ns) { spin_ns(ns); }
 
+/*
+ * Fused-producer stand-ins for tests: they store a part of a rank's partial the way a caller's own kernel
+ * would, with the device helpers of sifar_device.cuh (store_slot; plain stores + signal_block).
+ */
+template <int DT>
+__global__ void k_store_slots(const void *src, uint4 *slots, unsigned long long first, unsigned long long count,
+                              unsigned long long n, uint32_t tag)
+{
+    constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;
+    for (size_t s = first + (size_t)blockIdx.x * blockDim.x + threadIdx.x; s < first + count;
+         s += (size_t)gridDim.x * blockDim.x) {
+        uint32_t w[3] = {0u, 0u, 0u};
+        for (int k = 0; k < EPS && s * EPS + k < n; ++k) {
+            if (DT == SIFAR_BF16)
+                w[k >> 1] |= (uint32_t)reinterpret_cast<const uint16_t *>(src)[s * EPS + k] << ((k & 1) * 16);
+            else
+                w[k] = reinterpret_cast<const uint32_t *>(src)[s * EPS + k];
+        }
+        store_slot(slots, s, w[0], w[1], w[2], tag);
+    }
+}
+
+/* One CTA per flag block: plain 16-byte stores of the block's elements, then the block's flag. */
+template <int DT>
+__global__ void k_store_blocks(const void *src, void *dst, uint32_t *flags, unsigned long long stride_words,
+                               unsigned long long first, unsigned long long n, uint32_t tag)
+{
+    constexpr size_t EPV = (DT == SIFAR_BF16) ? 8 : 4;
+    const size_t esz = 16 / EPV;
+    const size_t b = first + blockIdx.x;
+    const size_t nvec = (size_t)n / EPV;
+    const size_t nblocks = nvec ? (nvec + kFlagBlockVecs - 1) / kFlagBlockVecs : 1;
+    for (size_t v = b * kFlagBlockVecs + threadIdx.x; v < (b + 1) * kFlagBlockVecs && v < nvec; v += blockDim.x)
+        st_slot(reinterpret_cast<uint4 *>(dst) + v, reinterpret_cast<const uint4 *>(src)[v]);
+    if (b == nblocks - 1)                           /* the ragged tail travels with the last block */
+        for (size_t i = nvec * EPV + threadIdx.x; i < (size_t)n; i += blockDim.x)
+            memcpy(reinterpret_cast<char *>(dst) + i * esz, reinterpret_cast<const char *>(src) + i * esz, esz);
+    signal_block(flags, (size_t)stride_words, b, tag);
+}
+
 /* ------------------------------------------------------------------------ */
 /* persistent chain kernel                                                   */
 /* ------------------------------------------------------------------------ */
@@ -313,9 +353,12 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
                 for (int r = 0; r < P; ++r) x[r] = ld_slot(src[r] + u);
                 if (MODE == SIFAR_SPECULATIVE) {
                     const unsigned before = reloads;
-                    if (!validate_slot<P>(x, src, u, e, a.timeout_ns, a.poll, reloads,
-                                          (TRACE && tracer && k == 0) ? a.trace + (size_t)s * kTraceSlots + 30 : nullptr)) {
-                        fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+                    const bool valid = validate_slot<P>(x, src, u, e, a.timeout_ns, a.poll, reloads,
+                                          (TRACE && tracer && k == 0) ? a.trace + (size_t)s * kTraceSlots + 30 : nullptr);
+                    /* the whole warp leaves together (its lanes have the same k and all have a unit): a lane that
+                       went on alone would meet the warp-wide vote of the next sentinel wait without its neighbours */
+                    if (!__all_sync(0xFFFFFFFFu, valid)) {
+                        if (!valid) fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
                         alive = false;
                         break;
                     }
@@ -546,6 +589,45 @@ struct sifar_chain {
     int grid;
     bool clustered;                 /* one thread-block cluster per chunk (placement only) */
 };
+
+/*
+ * Kernels that are launched for the first time while another kernel already waits for them must not be
+ * loaded by that launch: with lazy module loading a load can wait for the device to become idle.  The
+ * helpers that tests and benchmarks use to script orderings are loaded on the first call of any of them,
+ * the chain kernels when a chain is created.
+ */
+template <typename K>
+static cudaError_t preload(K kernel)
+{
+    cudaFuncAttributes at;
+    return cudaFuncGetAttributes(&at, kernel);
+}
+
+static cudaError_t preload_helpers()
+{
+    static cudaError_t done = [] {
+        cudaError_t e = preload(k_spin);
+        if (e == cudaSuccess) e = preload(k_store_slots<SIFAR_BF16>);
+        if (e == cudaSuccess) e = preload(k_store_slots<SIFAR_F32>);
+        if (e == cudaSuccess) e = preload(k_store_blocks<SIFAR_BF16>);
+        if (e == cudaSuccess) e = preload(k_store_blocks<SIFAR_F32>);
+        if (e == cudaSuccess) e = preload(k_probe<SIFAR_BF16>);
+        if (e == cudaSuccess) e = preload(k_probe<SIFAR_F32>);
+        if (e == cudaSuccess) e = preload(k_delays);
+        return e;
+    }();
+    return done;
+}
+
+template <int DT>
+static cudaError_t preload_produce()
+{
+    cudaError_t e = preload(k_produce<DT, SIFAR_BARRIER_ONESHOT>);
+    if (e == cudaSuccess) e = preload(k_produce<DT, SIFAR_DUALBUF>);
+    if (e == cudaSuccess) e = preload(k_produce<DT, SIFAR_SPECULATIVE>);
+    if (e == cudaSuccess) e = preload(k_produce<DT, kModeNoAllreduce>);
+    return e;
+}
 
 static bool valid_workload(const sifar_workload *w)
 {
@@ -782,6 +864,8 @@ extern "C" sifar_chain *sifar_chain_create(sifar_ctx *c, const sifar_workload *w
     cudaSetDevice(c->device);
     int rc = SIFAR_OK;
     auto setup = [&]() -> int {
+        SIFAR_CUDA(preload_helpers());
+        SIFAR_CUDA(c->dtype == SIFAR_BF16 ? preload_produce<SIFAR_BF16>() : preload_produce<SIFAR_F32>());
         if (impl == SIFAR_CHAIN_PERSISTENT) {
             int coop = 0;
             SIFAR_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
@@ -797,7 +881,7 @@ extern "C" sifar_chain *sifar_chain_create(sifar_ctx *c, const sifar_workload *w
         ch->concurrent = reduce_tiles(c, n, mode == kModeNoAllreduce ? SIFAR_DUALBUF : mode) <= kConcurrentTiles;
         ch->ev_step.assign((size_t)ch->steps, nullptr);
         for (int s = 0; s < ch->steps; ++s) SIFAR_CUDA(cudaEventCreateWithFlags(&ch->ev_step[s], cudaEventDisableTiming));
-        ch->launches_per_run = ch->steps * (c->P + (mode == kModeNoAllreduce ? 0 : reduce_launch_count(c, n, mode)));
+        ch->launches_per_run = ch->steps * (c->P + (mode == kModeNoAllreduce ? 0 : 1));      /* one reducer kernel per all-reduce */
         if (impl == SIFAR_CHAIN_GRAPH) {
             /* capture one run; every later replay finds the same parities because steps_per_run is even */
             cudaStream_t cap;
@@ -1010,10 +1094,57 @@ extern "C" int sifar_workload_delays(const sifar_workload *w, int P, unsigned t,
     return SIFAR_OK;
 }
 
+extern "C" int sifar_workload_preload(void)
+{
+    SIFAR_CUDA(preload_helpers());
+    SIFAR_CUDA(preload_produce<SIFAR_BF16>());
+    SIFAR_CUDA(preload_produce<SIFAR_F32>());
+    return SIFAR_OK;
+}
+
 extern "C" int sifar_spin(unsigned ns, void *stream)
 {
     if (ns > 50000000u) { set_error("sifar_spin: at most 50 ms"); return SIFAR_ERR_INVALID; }
+    SIFAR_CUDA(preload_helpers());
     k_spin<<<1, 1, 0, (cudaStream_t)stream>>>(ns);
+    SIFAR_CUDA(cudaGetLastError());
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_store_slots(const void *src, void *slots, size_t first_slot, size_t nslots, size_t n,
+                                 int dtype, unsigned tag, void *stream)
+{
+    if (!src || !slots || ((uintptr_t)slots & 15u) || (dtype != SIFAR_BF16 && dtype != SIFAR_F32)) {
+        set_error("sifar_store_slots: bad argument");
+        return SIFAR_ERR_INVALID;
+    }
+    if (nslots == 0) return SIFAR_OK;
+    SIFAR_CUDA(preload_helpers());
+    const unsigned grid = (unsigned)((nslots + 255) / 256 < 592 ? (nslots + 255) / 256 : 592);
+    if (dtype == SIFAR_BF16)
+        k_store_slots<SIFAR_BF16><<<grid, 256, 0, (cudaStream_t)stream>>>(src, (uint4 *)slots, first_slot, nslots, n, tag);
+    else
+        k_store_slots<SIFAR_F32><<<grid, 256, 0, (cudaStream_t)stream>>>(src, (uint4 *)slots, first_slot, nslots, n, tag);
+    SIFAR_CUDA(cudaGetLastError());
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_store_blocks(const void *src, void *dst, void *flags, size_t stride_words, size_t first_block,
+                                  size_t nblocks, size_t n, int dtype, unsigned tag, void *stream)
+{
+    if (!src || !dst || !flags || ((uintptr_t)src & 15u) || ((uintptr_t)dst & 15u) ||
+        (dtype != SIFAR_BF16 && dtype != SIFAR_F32) || nblocks > 0x7FFFFFFFu) {
+        set_error("sifar_store_blocks: bad argument");
+        return SIFAR_ERR_INVALID;
+    }
+    if (nblocks == 0) return SIFAR_OK;
+    SIFAR_CUDA(preload_helpers());
+    if (dtype == SIFAR_BF16)
+        k_store_blocks<SIFAR_BF16><<<(unsigned)nblocks, 256, 0, (cudaStream_t)stream>>>(src, dst, (uint32_t *)flags,
+                                                                                     stride_words, first_block, n, tag);
+    else
+        k_store_blocks<SIFAR_F32><<<(unsigned)nblocks, 256, 0, (cudaStream_t)stream>>>(src, dst, (uint32_t *)flags,
+                                                                                    stride_words, first_block, n, tag);
     SIFAR_CUDA(cudaGetLastError());
     return SIFAR_OK;
 }

@@ -17,3 +17,16 @@ def oracle():
     from oracle import oracle as o
     o.lib()
     return o
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _preloaded_helper_kernels():
+    """GPU runs: load the helper kernels before any test scripts a producer behind an already waiting reducer."""
+    try:
+        import torch
+        if torch.cuda.is_available():
+            from paper_2607_08973_b200 import binding as sf
+            sf.sifar_workload_preload()
+    except ImportError:
+        pass
+    yield

@@ -1,4 +1,4 @@
-"""Forced retries (the retry-latency experiment of Section 7, "Retry Overhead"): results do not
+"""Forced retries (the retry-latency experiment of Section 6.3, "Retry Overhead"): results do not
 change, the extra loads are counted, and the knob is refused outside its range."""
 import numpy as np
 import pytest

@@ -11,14 +11,6 @@ from gpu_util import BF16, F32, MODES, Ctx, assert_bits_equal, empty_out, out_to
 pytestmark = pytest.mark.gpu
 
 
-class RawDeviceArray:
-    """Wraps a raw device pointer so that torch can view it (CUDA array interface)."""
-
-    def __init__(self, ptr, nitems, typestr, itemsize):
-        self.__cuda_array_interface__ = {"shape": (nitems,), "typestr": typestr, "data": (ptr, False),
-                                         "version": 2, "strides": (itemsize,)}
-
-
 def _scripted(oracle, P, n, mode, delays_us, reducer_first, dtype=BF16, seed=7):
     """One call; rank r's pack is held back `delays_us[r]` microseconds behind a spin kernel on its stream."""
     with Ctx(P, n, dtype) as ctx:
@@ -127,36 +119,55 @@ def test_call_numbers_near_the_32_bit_limit(oracle, mode):
 
 
 def test_half_written_partial_then_the_rest(oracle):
-    """A fused producer that stores its slots itself: first half, a pause, second half."""
+    """A fused producer that stores its slots itself (device helper store_slot): first half, a pause, second half."""
     P, n = 4, 6 * 5000
     nslots = sf.sifar_slot_count(BF16, n)
     with Ctx(P, n, BF16) as ctx:
         xs = synth.rank_inputs(P, n, BF16, 21, "gauss")
+        xd = [to_device(x) for x in xs]
         out = empty_out(n, BF16)
-        images = []
-        for r in range(P):
-            ptr, epoch = sf.sifar_rank_buffer(ctx.h, r, sf.SPECULATIVE)
-            img = np.zeros((nslots, 4), dtype=np.uint32)
-            img[:, :3] = xs[r].view(np.uint32).reshape(nslots, 3)
-            img[:, 3] = epoch
-            # complex128 elements: torch moves each 16-byte slot image with one 16-byte access
-            src = torch.from_numpy(img.view(np.complex128).reshape(nslots).copy()).cuda()
-            dst = torch.as_tensor(RawDeviceArray(ptr, nslots, "<c16", 16), device="cuda")
-            images.append((src, dst))
+        where = [sf.sifar_rank_buffer(ctx.h, r, sf.SPECULATIVE) for r in range(P)]
         ps = [torch.cuda.Stream() for _ in range(P)]
         rs = torch.cuda.Stream()
         torch.cuda.synchronize()
         half = nslots // 2
         sf.sifar_allreduce(ctx.h, None, out.data_ptr(), n, sf.SPECULATIVE, rs.cuda_stream)
-        for r, (src, dst) in enumerate(images):
-            with torch.cuda.stream(ps[r]):
-                sf.sifar_spin(20_000, ps[r].cuda_stream)
-                dst[:half].copy_(src[:half])
-                sf.sifar_spin(100_000, ps[r].cuda_stream)
-                dst[half:].copy_(src[half:])
+        for r, (ptr, epoch) in enumerate(where):                # the slot stores take tag and address as arguments
+            sf.sifar_spin(20_000, ps[r].cuda_stream)
+            sf.sifar_store_slots(xd[r].data_ptr(), ptr, 0, half, n, BF16, epoch, ps[r].cuda_stream)
+            sf.sifar_spin(100_000, ps[r].cuda_stream)
+            sf.sifar_store_slots(xd[r].data_ptr(), ptr, half, nslots - half, n, BF16, epoch, ps[r].cuda_stream)
         torch.cuda.synchronize()
         assert sf.sifar_status(ctx.h) == 0
         got, _ = out_to_numpy(out, n, BF16)
         assert_bits_equal(got, oracle.allreduce(xs, BF16), BF16, "half-written")
         st = sf.sifar_get_stats(ctx.h)
         assert st["calls_with_retry"] == 1 and st["slot_reloads"] > 0
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_a_producer_that_is_not_ordered_after_the_previous_call_is_refused(oracle, mode):
+    """The producer of call e + 1 must be ordered after the reducer of call e (it takes the call number from
+    device memory).  One that runs too early finds the number one short: SIFAR_ERR_EPOCH, in every mode, no hang."""
+    P, n = 2, 4096
+    with Ctx(P, n, BF16, timeout_us=20_000) as ctx:
+        xs = synth.rank_inputs(P, n, BF16, 3, "gauss")
+        xd = [to_device(x) for x in xs]
+        out = empty_out(n, BF16)
+        rs, ps = torch.cuda.Stream(), torch.cuda.Stream()
+        for r in range(P):
+            sf.sifar_pack(ctx.h, r, xd[r].data_ptr(), n, mode, ps.cuda_stream)
+        torch.cuda.synchronize()
+        sf.sifar_spin(3_000_000, rs.cuda_stream)              # the reducer of call 1 is held back 3 ms ...
+        sf.sifar_allreduce(ctx.h, None, out.data_ptr(), n, mode, rs.cuda_stream)
+        sf.sifar_pack(ctx.h, 0, xd[0].data_ptr(), n, mode, ps.cuda_stream)   # ... the producer of call 2 is not
+        ps.synchronize()
+        assert sf.sifar_status(ctx.h) == sf.ERR_EPOCH
+        torch.cuda.synchronize()
+        sf.sifar_reset(ctx.h, 0)
+        for r in range(P):
+            sf.sifar_pack(ctx.h, r, xd[r].data_ptr(), n, mode, ps.cuda_stream)
+        sf.sifar_allreduce(ctx.h, None, out.data_ptr(), n, mode, rs.cuda_stream)
+        torch.cuda.synchronize()
+        got, _ = out_to_numpy(out, n, BF16)
+        assert_bits_equal(got, oracle.allreduce(xs, BF16), BF16, "after reset")

@@ -394,3 +394,41 @@ def test_chain_is_composition_of_steps(oracle):
     # resuming in the middle gives the same tail
     tail = oracle.chain(w, P, n, BF16, 3, t0=4, out_prev=outs[2])
     np.testing.assert_array_equal(tail, outs[3:6])
+
+
+def test_fp32_chain_is_composition_of_steps_and_follows_the_float64_route(oracle):
+    """The fp32 branch of the chain: every step equals the all-reduce of the ranks' next partials, a run resumed in
+    the middle gives the same tail, and the whole chain is re-derived here through float64 (every product, the
+    sum of the update and every rank-order add rounded to binary32 separately), which shares nothing with the C code."""
+    P, n, steps = 3, 257, 7
+    w = oracle.Workload(oracle.KIND_UNIFORM, 0x5EED0004, 1.0 / 3.0, 0.5, 0, 0)
+    outs = oracle.chain(w, P, n, F32, steps)
+    assert outs.dtype == np.float32 and outs.shape == (steps, n)
+    prev = None
+    for s in range(steps):
+        xs = [oracle.workload_first(w, r, n, F32) if s == 0 else oracle.workload_next(w, r, s + 1, prev, F32)
+              for r in range(P)]
+        prev = oracle.allreduce(xs, F32)
+        np.testing.assert_array_equal(outs[s].view(np.uint32), prev.view(np.uint32))
+    tail = oracle.chain(w, P, n, F32, 3, t0=5, out_prev=outs[3])
+    np.testing.assert_array_equal(tail.view(np.uint32), outs[4:7].view(np.uint32))
+    # float64 route: binary32 products and sums are exact in binary64, so one rounding each reproduces them
+    i = np.arange(n, dtype=np.uint32)
+    f32, f64 = np.float32, np.float64
+    prev = None
+    for s in range(steps):
+        t = s + 1
+        xs = []
+        for r in range(P):
+            z = synth.uniform(0x5EED0004, r, t, i)
+            if prev is None:
+                xs.append(z.astype(f32))
+            else:
+                a = (prev.astype(f64) * f64(f32(1.0 / 3.0))).astype(f32)
+                b = (z.astype(f64) * f64(f32(0.5))).astype(f32)
+                xs.append((a.astype(f64) + b.astype(f64)).astype(f32))
+        acc = xs[0]
+        for r in range(1, P):
+            acc = (acc.astype(f64) + xs[r].astype(f64)).astype(f32)
+        np.testing.assert_array_equal(outs[s].view(np.uint32), acc.view(np.uint32))
+        prev = acc
