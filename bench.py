@@ -40,8 +40,10 @@ sys.path.insert(0, ROOT)
 METRIC = "p50 us per P=8 emulated all-reduce (decode payload), with HBM roofline fraction at a 16 MiB payload"
 P, HIDDEN, ARS_PER_STEP = 8, 4096, 64
 LARGE_N = 8 << 20                      # 16 MiB of bf16 per rank
-# DRAM bytes per launch of k_reduce_spec<bf16,8> at LARGE_N from one ncu capture: 179.00 MB read + 12.66 MB written
-NCU_TRAFFIC_BYTES = 191_657_728
+NOMINAL_GBS = 8000.0                   # the HBM3e figure the metric names
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the roofline kernel at LARGE_N, from the
+# ncu capture summarised in the file named below; refreshed whenever the reducer kernels change
+NCU_TRAFFIC = {"bytes": None, "captured_at_commit": None, "summary": None}
 
 
 def read_peaks() -> tuple[float, str]:
@@ -125,6 +127,23 @@ def oracle_allreduce_us(oracle, synth, n: int, budget_s: float) -> tuple[float, 
     return float(np.median(times) * 1e6), len(times)
 
 
+def oracle_allreduce_all_cores(oracle, xs, cores: int) -> np.ndarray:
+    """The oracle as it stands on every host core: the elements are independent, so [0, n) is cut into one range
+    per core and each thread runs the unchanged single-threaded loop on its range (ctypes releases the GIL)."""
+    from concurrent.futures import ThreadPoolExecutor
+    n = xs[0].size
+    cuts = [n * k // cores for k in range(cores + 1)]
+    out = np.empty_like(xs[0])
+
+    def work(k):
+        a, b = cuts[k], cuts[k + 1]
+        if b > a:
+            out[a:b] = oracle.allreduce([x[a:b] for x in xs], 0)
+    with ThreadPoolExecutor(max_workers=cores) as pool:
+        list(pool.map(work, range(cores)))
+    return out
+
+
 def run_reference(args) -> None:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -140,7 +159,7 @@ def run_reference(args) -> None:
     line = {
         "impl": "reference", "metric": METRIC, "value": per_ar, "unit": "us", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "accumulator": "f32", "data": "synthetic",
         "config": {"workload": "config2 llama-shaped decode step: P=8, n=4096 bf16, 64 dependent all-reduces, "
                                "seeded elementwise producers (CPU oracle, one thread)"},
         "cpu_baseline": {"value": per_ar, "unit": "us", "cores": 1, "kind": "oracle",
@@ -294,7 +313,8 @@ def measure_pack(sf, torch, P_, n, mode, reps=8):
         main.synchronize()
         ts.append(ev0.elapsed_time(ev1) * 1e-3)
     sf.sifar_destroy(ctx)
-    per_rank = n * 2 + (sf.sifar_slot_count(0, n) * 16 if mode == sf.SPECULATIVE else n * 2)
+    slots = mode == sf.SPECULATIVE and sf.sifar_spec_format(P_, 0, n) == sf.FORMAT_SLOTS
+    per_rank = n * 2 + (sf.sifar_slot_count(0, n) * 16 if slots else n * 2)
     return float(np.median(ts[2:])), P_ * per_rank
 
 
@@ -315,6 +335,59 @@ def measure_e2e(sf, torch, synth, n, mode, warmup, steps):
     return np.asarray(per_call) * 1e6
 
 
+def rates(sf, P_, dtype, n, mode, seconds, peak_gbs):
+    """Both rates of one reducer launch: algorithmic traffic (reads of the partials in the format of the mode,
+    the write of the result, the flag words) and payload-effective (P + 1) * n * s, each over the launch time."""
+    alg = sf.sifar_algorithmic_bytes(P_, dtype, n, mode)
+    payload = (P_ + 1) * n * (2 if dtype == 0 else 4)
+    gbs = alg / seconds / 1e9
+    r = {"us": round(seconds * 1e6, 2), "algorithmic_bytes": alg, "GBps": round(gbs, 1),
+         "frac": round(gbs / peak_gbs, 4), "frac_of_8TBs_nominal": round(gbs / NOMINAL_GBS, 4),
+         "payload_GBps": round(payload / seconds / 1e9, 1),
+         "payload_frac_of_8TBs_nominal": round(payload / seconds / 1e9 / NOMINAL_GBS, 4)}
+    if mode == sf.SPECULATIVE:
+        r["format"] = "tiles" if sf.sifar_spec_format(P_, dtype, n) == sf.FORMAT_TILES else "slots"
+    if gbs > peak_gbs:
+        r["note"] = "above the measured copy bandwidth: the peak is a read+write copy, this kernel reads 8 bytes per byte written"
+    return r
+
+
+def reducer_points(sf, torch, peak_gbs, points, iters=4, max_ctx=24):
+    """Reducer alone on ready data, one row per (P, n, dtype): every mode, both rates.  Contexts per timed
+    region: enough that the partials exceed twice the L2 and that the cost of an event pair is spread thin."""
+    rows = []
+    for P_, n, dtype in points:
+        per_ctx = P_ * n * (2 if dtype == 0 else 4)
+        nctx = int(min(max_ctx, max(min(6, max_ctx), (20 << 30) // max(3 * per_ctx, 1))))
+        row = {"P": P_, "n": n, "dtype": "bf16" if dtype == 0 else "f32",
+               "payload_bytes_per_rank": n * (2 if dtype == 0 else 4), "launches_per_timed_region": nctx}
+        for mode in (sf.BARRIER_ONESHOT, sf.DUALBUF, sf.SPECULATIVE):
+            mean_s, med_s, _ = measure_roofline(sf, torch, P_, n, mode, 2, iters, dtype=dtype, nctx=nctx)
+            row[sf.MODE_NAMES[mode]] = rates(sf, P_, dtype, n, mode, med_s, peak_gbs)
+        rows.append(row)
+    return rows
+
+
+def measure_skew(sf, torch, synth, runs=6):
+    """Config 5: P = 8, n = 16384 integers, seeded 0-20 us producer delays; persistent chain with one reader and
+    with P readers, speculative mode: intervals and the retry counters."""
+    n, steps = 16384, 100
+    c = Chain(sf, torch, synth, n, sf.SPECULATIVE, sf.CHAIN_PERSISTENT, steps=steps, name="skew")
+    for _ in range(2):
+        c.run()
+    c.stream.synchronize()
+    base = sf.sifar_get_stats(c.ctx)
+    iv = c.intervals_us(runs)
+    st = sf.sifar_get_stats(c.ctx)
+    calls = st["calls"] - base["calls"]
+    one = {"p50_us": round(pct(iv, 50), 3), "p99_us": round(pct(iv, 99), 3), "calls": calls,
+           "calls_with_retry": st["calls_with_retry"] - base["calls_with_retry"],
+           "slot_reloads": st["slot_reloads"] - base["slot_reloads"]}
+    c.close()
+    sym = measure_symmetric(sf, torch, synth, P, n, name="skew", steps=steps, warm=2, runs=runs)
+    return {"one_reader_persistent_speculative": one, "p_readers": sym}
+
+
 def payload_sweep(sf, torch, exps=range(10, 26), ranks=(2, 4, 8)):
     """Config 4: reducer time against payload, data ready, every mode; bf16 for all P, fp32 for P = 8.
 
@@ -328,14 +401,12 @@ def payload_sweep(sf, torch, exps=range(10, 26), ranks=(2, 4, 8)):
             for ex in exps:
                 n = 1 << ex
                 per_call = P_ * n * (2 if dtype == 0 else 4)
-                nctx = int(min(24, max(4, (2 * 126e6) // max(per_call, 1) + 1)))
+                nctx = int(min(24, max(6, (20 << 30) // max(3 * per_call, 1))))
                 row = {"P": P_, "dtype": "bf16" if dtype == 0 else "f32", "n": n,
                        "payload_bytes_per_rank": n * (2 if dtype == 0 else 4)}
                 for mode in (sf.BARRIER_ONESHOT, sf.DUALBUF, sf.SPECULATIVE):
                     mean_s, med_s, _ = measure_roofline(sf, torch, P_, n, mode, 2, 5, dtype=dtype, nctx=nctx)
-                    alg = sf.sifar_algorithmic_bytes(P_, dtype, n, mode)
-                    row[sf.MODE_NAMES[mode]] = {"us": round(med_s * 1e6, 2), "GBps": round(alg / med_s / 1e9, 1)}
-                row["speculative"]["format"] = "tiles" if sf.sifar_spec_format(P_, dtype, n) == sf.FORMAT_TILES else "slots"
+                    row[sf.MODE_NAMES[mode]] = rates(sf, P_, dtype, n, mode, med_s, read_peaks()[0])
                 rows.append(row)
     return rows
 
@@ -432,7 +503,7 @@ def run_gpu(args) -> None:
         stats = sf.sifar_get_stats(main.ctx)
         main.close()
 
-    detail, roof, roof_decode, e2e, cpu = {}, None, None, None, None
+    detail, roof, roof_decode, e2e, cpu, by_payload = {}, None, None, None, None, None
     if rank == 0 and args.only == "p_readers":
         detail["p_readers"] = {"llama P=8 8KB": measure_symmetric(sf, torch, synth, P, n, warm=args.warmup,
                                                                  runs=max(1, args.steps))}
@@ -441,10 +512,22 @@ def run_gpu(args) -> None:
         w0 = time.time()
         modes = (sf.BARRIER_ONESHOT, sf.DUALBUF, sf.SPECULATIVE, sf.CHAIN_NO_ALLREDUCE)
         impls = (sf.CHAIN_PERSISTENT,) if args.skip_graph else (sf.CHAIN_PERSISTENT, sf.CHAIN_GRAPH)
+        reps = max(8, args.steps // 8)
         if args.only == "all":
-            detail["modes"] = measure_modes(sf, torch, synth, n, args.warmup, max(8, args.steps // 8), impls, modes)
-        if args.only == "all":
+            detail["modes"] = measure_modes(sf, torch, synth, n, args.warmup, reps, impls, modes)
             detail["p_readers"] = {"llama P=8 8KB": measure_symmetric(sf, torch, synth, P, n)}
+            # -- 2b. the metric is a curve: the same step against the payload, in the default run ---
+            by_payload = {
+                "llama_step_by_batch_tokens": {"1": detail["modes"]},
+                "moe_step_by_batch_tokens": {},
+            }
+            for b in (4, 16):
+                by_payload["llama_step_by_batch_tokens"][str(b)] = measure_modes(
+                    sf, torch, synth, HIDDEN * b, 5, max(8, reps // 4), impls, modes, rounds=2)
+            for b in (1, 8, 32):
+                by_payload["moe_step_by_batch_tokens"][str(b)] = measure_modes(
+                    sf, torch, synth, HIDDEN * b, 3, 6, impls, modes, rounds=2, name="moe", steps=120)
+            by_payload["skewed_arrival_config5"] = measure_skew(sf, torch, synth)
         if args.sweep and args.only == "all":
             for P_ in (2, 4, 8):
                 for kb in (8, 16, 32):
@@ -452,7 +535,7 @@ def run_gpu(args) -> None:
                         detail["p_readers"][f"llama P={P_} {kb}KB"] = measure_symmetric(sf, torch, synth, P_, kb * 512)
                 detail["p_readers"][f"skew P={P_} 32KB"] = measure_symmetric(sf, torch, synth, P_, 16384, name="skew", runs=4)
             detail["by_batch_tokens"] = {
-                str(b): measure_modes(sf, torch, synth, HIDDEN * b, args.warmup, max(8, args.steps // 8),
+                str(b): measure_modes(sf, torch, synth, HIDDEN * b, args.warmup, reps,
                                       (sf.CHAIN_PERSISTENT, sf.CHAIN_GRAPH), modes)
                 for b in (2, 4, 8, 16)}
             # config 3: MoE-shaped step, 120 dependent all-reduces, 1 % outliers
@@ -463,32 +546,38 @@ def run_gpu(args) -> None:
             detail["streams"] = measure_modes(sf, torch, synth, n, 3, 8, (sf.CHAIN_STREAMS,), modes, rounds=2)
             detail["payload_sweep"] = payload_sweep(sf, torch)
             detail["retry_overhead"] = retry_overhead(sf, torch, synth)
-        # -- 3. roofline: 16 MiB per rank, inputs larger than L2 -------------------------------------
-        r_iters = max(5, min(20, args.steps))
-        mean_s, med_s, cnt = measure_roofline(sf, torch, P, LARGE_N, sf.SPECULATIVE, 3, r_iters)
-        alg = sf.sifar_algorithmic_bytes(P, sf.BF16, LARGE_N, sf.SPECULATIVE)
-        roof = {"bound": "hbm", "achieved": round(alg / mean_s / 1e9, 1), "peak": peak_gbs, "unit": "GB/s",
-                "frac": round(alg / mean_s / 1e9 / peak_gbs, 4), "peak_kind": f"of {peak_kind}", "traffic": None,
-                "kernel": "k_reduce_spec<bf16,P=8>", "workload": "config4 P=8 n=8Mi bf16 (16 MiB/rank), speculative, 6 rotating contexts (1.2 GB of partials >> L2)",
-                "algorithmic_bytes": alg, "kernel_us": round(mean_s * 1e6, 2), "launches_timed": cnt,
-                "frac_of_8TBs_nominal": round(alg / mean_s / 1e9 / 8000.0, 4)}
-        others = {}
-        for m in (sf.BARRIER_ONESHOT, sf.DUALBUF):
-            ms_, _, _ = measure_roofline(sf, torch, P, LARGE_N, m, 2, r_iters)
-            ab = sf.sifar_algorithmic_bytes(P, sf.BF16, LARGE_N, m)
-            others[sf.MODE_NAMES[m]] = {"kernel_us": round(ms_ * 1e6, 2), "achieved": round(ab / ms_ / 1e9, 1),
-                                        "frac": round(ab / ms_ / 1e9 / peak_gbs, 4)}
-        roof["other_modes"] = others
-        ms_, _, _ = measure_roofline(sf, torch, P, 4 * LARGE_N, sf.SPECULATIVE, 2, max(3, r_iters // 3), nctx=3)
-        ab = sf.sifar_algorithmic_bytes(P, sf.BF16, 4 * LARGE_N, sf.SPECULATIVE)
-        roof["at_64MiB_per_rank"] = {"kernel_us": round(ms_ * 1e6, 2), "achieved": round(ab / ms_ / 1e9, 1),
-                                     "frac": round(ab / ms_ / 1e9 / peak_gbs, 4)}
+        # -- 3. reducer alone against the payload; the roofline kernel is the 16 MiB point ------------
+        r_iters = max(4, min(10, args.steps))
+        points = [(P, LARGE_N, 0)]
+        if args.only == "all":
+            points = [(P, 1 << 10, 0), (P, 1 << 19, 0), (P, LARGE_N, 0), (P, 4 * LARGE_N, 0), (P, LARGE_N // 2, 1)]
+        rows = reducer_points(sf, torch, peak_gbs, points, iters=r_iters, max_ctx=args.roofline_contexts)
+        big = next(r for r in rows if r["n"] == LARGE_N and r["dtype"] == "bf16")
+        sp = big["speculative"]
+        roof = {"bound": "hbm", "achieved": sp["GBps"], "peak": peak_gbs, "unit": "GB/s", "frac": sp["frac"],
+                "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC["bytes"],
+                "traffic_source": NCU_TRAFFIC,
+                "kernel": "k_reduce_plain<bf16,P=8,flagged tiles> (speculative mode at this size)",
+                "workload": f"config4 P=8 n=8Mi bf16 (16 MiB/rank), speculative, {big['launches_per_timed_region']} "
+                            "contexts back to back (partials >> L2); producers on their own streams, complete "
+                            "before the timed region",
+                "algorithmic_bytes": sp["algorithmic_bytes"], "kernel_us": sp["us"],
+                "launches_timed": big["launches_per_timed_region"] * r_iters,
+                "frac_of_8TBs_nominal": sp["frac_of_8TBs_nominal"],
+                "payload_effective": {"GBps": sp["payload_GBps"], "frac_of_8TBs_nominal": sp["payload_frac_of_8TBs_nominal"],
+                                      "what": "(P + 1) * n * 2 bytes over the same launch time"},
+                "other_modes": {k: big[k] for k in ("barrier_oneshot", "dualbuf")}}
+        if sp["frac"] > 1.0:
+            roof["peak_note"] = "frac above 1: the measured peak is a read+write copy and understates a read-dominated kernel"
+        big64 = [r for r in rows if r["n"] == 4 * LARGE_N]
+        if big64:
+            roof["at_64MiB_per_rank"] = {k: big64[0][k] for k in ("barrier_oneshot", "dualbuf", "speculative")}
+        if by_payload is not None:
+            by_payload["reducer_alone"] = rows
         pk_s, pk_bytes = measure_pack(sf, torch, P, LARGE_N, sf.SPECULATIVE)
-        roof["producer_store"] = {"kernel": "k_pack<bf16,speculative> x 8 ranks on 8 streams", "us": round(pk_s * 1e6, 1),
+        roof["producer_store"] = {"kernel": "k_pack<bf16, flagged tiles> x 8 ranks on 8 streams", "us": round(pk_s * 1e6, 1),
                                   "bytes": pk_bytes, "achieved": round(pk_bytes / pk_s / 1e9, 1),
                                   "frac": round(pk_bytes / pk_s / 1e9 / peak_gbs, 4)}
-        roof["traffic"] = NCU_TRAFFIC_BYTES
-        roof["traffic_source"] = "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel and size"
         alg_d = sf.sifar_algorithmic_bytes(P, sf.BF16, n, sf.SPECULATIVE) * ARS_PER_STEP
         step_s = secs / args.steps if secs else float("inf")
         roof_decode = {"bound": "latency", "kernel": "k_chain<bf16,P=8,speculative>", "achieved": round(alg_d / step_s / 1e9, 1),
@@ -507,40 +596,55 @@ def run_gpu(args) -> None:
                        "a stream synchronisation; per call"}
         # -- 5. CPU oracle ---------------------------------------------------------------------------
         from oracle import oracle
-        ar_us, reps = oracle_allreduce_us(oracle, synth, n, 6.0)
+        ar_us, reps_ar = oracle_allreduce_us(oracle, synth, n, 5.0)
         t0 = time.perf_counter()
         nsteps = 0
-        while time.perf_counter() - t0 < 8.0:
+        while time.perf_counter() - t0 < 7.0:
             oracle_decode_step_seconds(oracle, synth, n, ARS_PER_STEP)
             nsteps += 1
         chain_us = (time.perf_counter() - t0) / (nsteps * ARS_PER_STEP) * 1e6
-        big = synth.rank_inputs(P, 1 << 20, 0, 5, "uniform")
+        cores = os.cpu_count() or 1
+        big_xs = synth.rank_inputs(P, 1 << 22, 0, 5, "uniform")
         t0 = time.perf_counter()
-        oracle.allreduce(big, 0)
+        one = oracle.allreduce(big_xs, 0)
         big_s = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        many = oracle_allreduce_all_cores(oracle, big_xs, cores)
+        all_s = time.perf_counter() - t0
+        assert np.array_equal(one, many), "the oracle on all cores differs from the oracle on one"
+        big_bytes = sf.sifar_algorithmic_bytes(P, 0, 1 << 22, sf.DUALBUF)
         cpu = {"value": round(chain_us, 2), "unit": "us", "cores": 1, "kind": "oracle",
-               "sample": f"{nsteps} decode steps (64 chained all-reduces each, seeded producers included) in 8 s; "
-                         f"the all-reduce alone: {ar_us:.1f} us p50 over {reps} calls; P=8 n=1Mi: "
-                         f"{sf.sifar_algorithmic_bytes(P, 0, 1 << 20, sf.DUALBUF) / big_s / 1e9:.2f} GB/s",
-               "allreduce_only_us": round(ar_us, 2), "host_cores_available": os.cpu_count()}
+               "sample": f"{nsteps} decode steps (64 chained all-reduces each, seeded producers included) in 7 s on "
+                         f"one core; the all-reduce alone: {ar_us:.1f} us p50 over {reps_ar} calls",
+               "allreduce_only_us": round(ar_us, 2), "host_cores_available": cores,
+               "large_payload": {"P": P, "n": 1 << 22, "bytes": big_bytes,
+                                 "one_core": {"seconds": round(big_s, 4), "GBps": round(big_bytes / big_s / 1e9, 2)},
+                                 "all_cores": {"cores": cores, "seconds": round(all_s, 4),
+                                               "GBps": round(big_bytes / all_s / 1e9, 2),
+                                               "bit_identical_to_one_core": True,
+                                               "how": "the unchanged oracle loop on one element range per thread"}}}
 
     clocks = sampler.stop(windows)
     if rank == 0:
         line = {
             "metric": METRIC, "value": round(p50, 3), "unit": "us", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(secs / args.steps * 1e3, 5), "higher_is_better": False,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "accumulator": "f32", "data": "synthetic",
             "config": {"workload": "config2 llama-shaped decode step: P=8, n=4096 bf16 (8 KB/rank), 64 dependent "
                                    "all-reduces per step, seeded elementwise producers, speculative mode, "
                                    "persistent chain kernel",
                        "l2": "decode payloads are L2-resident by design (fresh partials every step); the roofline "
-                             "section uses inputs larger than L2 (6 rotating contexts, 1.2 GB of partials)",
+                             "section uses inputs larger than L2 (24 contexts back to back, 3.6 GB of partials)",
                        "replicas": world},
             "p99_us": round(p99, 3), "us_per_allreduce_mean": round(secs / args.steps / ARS_PER_STEP * 1e6, 3),
             "roofline": roof, "roofline_decode": roof_decode, "cpu_baseline": cpu, "e2e": e2e,
+            "by_payload": by_payload,
             "gpu_launches": launches, "clocks": clocks,
             "speculation": {"calls": stats["calls"], "misspeculated": stats["calls_with_retry"],
-                            "slot_reloads": stats["slot_reloads"]},
+                            "slot_reloads": stats["slot_reloads"],
+                            "note": "one reader: the reducer always runs ahead of the producers it feeds, so every "
+                                    "call re-loads; the rate that means what it means in the paper is per rank in "
+                                    "detail.p_readers and by_payload.skewed_arrival_config5.p_readers"},
             "detail": detail,
             "paper_context": "8xH200: oneshot 8 KB TP8 transfer 4.01 us; best baseline 5.11 us -> SiFAR 2.44 us "
                              "(with in-switch redundant pull, not built here)",
@@ -559,6 +663,9 @@ def main() -> None:
     ap.add_argument("--only", default="all", choices=["all", "decode", "roofline", "p_readers"],
                     help="profiling aid: run the timed decode region only, the roofline section only, or the "
                          "P-reader chain only")
+    ap.add_argument("--roofline-contexts", type=int, default=24,
+                    help="profiling aid: contexts (launches) per timed region of the reducer-alone section; a capture "
+                         "under ncu wants few (each holds 0.6 GB at 16 MiB per rank)")
     ap.add_argument("--skip-graph", action="store_true",
                     help="profiling aid: leave out the graph / stream chains (under ncu kernels are serialised, and "
                          "those chains' reducers wait for producers that run concurrently)")
