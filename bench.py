@@ -412,34 +412,67 @@ def payload_sweep(sf, torch, exps=range(10, 26), ranks=(2, 4, 8)):
     return rows
 
 
+def _sym_run(sf, torch, synth, ranks, n, mode, name, steps, warm, runs, forced=0):
+    d = synth.chain_workload(name, ranks)
+    ctx = sf.sifar_create(ranks, n, 0)
+    if forced:
+        sf.sifar_debug_force_retries(ctx, forced)
+    stride = sf.sifar_chain_ring_stride(0, n)
+    rings = torch.zeros(ranks * 2 * stride, dtype=torch.uint8, device="cuda")
+    ch = sf.sifar_symchain_create(ctx, sf.make_workload(**d), n, mode, rings.data_ptr(), 2, steps)
+    iv = []
+    for i in range(warm + runs):
+        sf.sifar_symchain_run(ch, 0)
+        if i >= warm:
+            st = np.array(sf.sifar_symchain_stamps(ch, steps), dtype=np.int64)
+            iv.append(np.diff(st)[1:] * 1e-3)
+    iv = np.concatenate(iv)
+    r = {"p50_us": round(pct(iv, 50), 3), "p99_us": round(pct(iv, 99), 3)}
+    if mode in (sf.SPECULATIVE, sf.SYMCHAIN_FLAGVAL, sf.SYMCHAIN_FLAGVAL_ORDERED):
+        rt = sf.sifar_symchain_retries(ch, ranks)
+        stt = sf.sifar_get_stats(ctx)
+        r["misspeculated_steps_per_rank"] = [round(x / ((warm + runs) * steps), 3) for x in rt]
+        r["slot_reloads_per_call"] = round(stt["slot_reloads"] / max(1, stt["calls"]), 1)
+    sf.sifar_symchain_destroy(ch)
+    sf.sifar_destroy(ctx)
+    return r
+
+
+SYM_NAMES = {4: "twoshot", 3: "no_allreduce", 5: "flagval_paper", 6: "flagval_ordered", 7: "unchecked_pull",
+             0: "barrier_oneshot", 1: "dualbuf", 2: "speculative"}
+
+
 def measure_symmetric(sf, torch, synth, ranks, n, name="llama", steps=ARS_PER_STEP, warm=3, runs=8):
     """The chain with P readers (every rank reduces for itself): p50 / p99 us between complete results on all
-    ranks, every mode and the floor without all-reduce; mis-speculation per rank for the speculative mode."""
-    d = synth.chain_workload(name, ranks)
+    ranks, every mode and the floor without all-reduce; mis-speculation per rank for the validating modes.
+    flagval_paper = the paper's per-threadblock validation flag pulled together with the payload,
+    flagval_ordered = the same with the payload pulled after the flags, unchecked_pull = no validation at all
+    (timing floor; its results are not a sum)."""
     res = {}
-    names = {sf.SYMCHAIN_TWOSHOT: "twoshot", sf.CHAIN_NO_ALLREDUCE: "no_allreduce", **sf.MODE_NAMES}
-    for mode in (sf.BARRIER_ONESHOT, sf.SYMCHAIN_TWOSHOT, sf.DUALBUF, sf.SPECULATIVE, sf.CHAIN_NO_ALLREDUCE):
-        ctx = sf.sifar_create(ranks, n, 0)
-        stride = sf.sifar_chain_ring_stride(0, n)
-        rings = torch.zeros(ranks * 2 * stride, dtype=torch.uint8, device="cuda")
-        ch = sf.sifar_symchain_create(ctx, sf.make_workload(**d), n, mode, rings.data_ptr(), 2, steps)
-        iv = []
-        for i in range(warm + runs):
-            sf.sifar_symchain_run(ch, 0)
-            if i >= warm:
-                st = np.array(sf.sifar_symchain_stamps(ch, steps), dtype=np.int64)
-                iv.append(np.diff(st)[1:] * 1e-3)
-        iv = np.concatenate(iv)
-        r = {"p50_us": round(pct(iv, 50), 3), "p99_us": round(pct(iv, 99), 3)}
-        if mode == sf.SPECULATIVE:
-            rt = sf.sifar_symchain_retries(ch, ranks)
-            stt = sf.sifar_get_stats(ctx)
-            r["misspeculated_steps_per_rank"] = [round(x / ((warm + runs) * steps), 3) for x in rt]
-            r["slot_reloads_per_call"] = round(stt["slot_reloads"] / max(1, stt["calls"]), 1)
-        res[names[mode]] = r
-        sf.sifar_symchain_destroy(ch)
-        sf.sifar_destroy(ctx)
+    for mode in (sf.BARRIER_ONESHOT, sf.SYMCHAIN_TWOSHOT, sf.DUALBUF, sf.SYMCHAIN_FLAGVAL_ORDERED, sf.SYMCHAIN_FLAGVAL,
+                 sf.SPECULATIVE, sf.SYMCHAIN_UNCHECKED, sf.CHAIN_NO_ALLREDUCE):
+        res[SYM_NAMES[mode]] = _sym_run(sf, torch, synth, ranks, n, mode, name, steps, warm, runs)
     return res
+
+
+def verification_overhead(sf, torch, synth, shapes=((8, 4096), (8, 16384), (2, 4096)), forced=(1, 2, 3)):
+    """Section 6.3, "Mis-Speculation and Verification Overhead" and "Retry Overhead", in the chain with P readers:
+    p50 per all-reduce of the two validation schemes (the paper's per-threadblock flags, tags inside the slots)
+    over the same pull without any validation, and what each forced retry adds to either."""
+    out = {}
+    for P_, n in shapes:
+        run = lambda mode, k=0: _sym_run(sf, torch, synth, P_, n, mode, "llama", ARS_PER_STEP, 3, 6, forced=k)["p50_us"]
+        base = run(sf.SYMCHAIN_UNCHECKED)
+        row = {"unchecked_pull_p50_us": base, "no_allreduce_p50_us": run(sf.CHAIN_NO_ALLREDUCE),
+               "barrier_oneshot_p50_us": run(sf.BARRIER_ONESHOT)}
+        for key, mode in (("flagval_paper", sf.SYMCHAIN_FLAGVAL), ("flagval_ordered", sf.SYMCHAIN_FLAGVAL_ORDERED),
+                          ("slot_tags", sf.SPECULATIVE)):
+            p50 = run(mode)
+            row[key] = {"p50_us": p50, "over_unchecked_us": round(p50 - base, 3)}
+            if mode != sf.SYMCHAIN_FLAGVAL_ORDERED:
+                row[key]["forced_retries_p50_us"] = {str(k): run(mode, k) for k in forced}
+        out[f"P{P_}_{n * 2 // 1024}KB"] = row
+    return out
 
 
 def retry_overhead(sf, torch, synth, ranks=(2, 4, 8), kbytes=(8, 16, 32), forced=(0, 1, 2, 3)):
@@ -529,6 +562,7 @@ def run_gpu(args) -> None:
                 by_payload["moe_step_by_batch_tokens"][str(b)] = measure_modes(
                     sf, torch, synth, HIDDEN * b, 3, 6, impls, modes, rounds=2, name="moe", steps=120)
             by_payload["skewed_arrival_config5"] = measure_skew(sf, torch, synth)
+            detail["verification_overhead"] = verification_overhead(sf, torch, synth)
         if args.sweep and args.only == "all":
             for P_ in (2, 4, 8):
                 for kb in (8, 16, 32):

@@ -76,6 +76,22 @@ enum { SIFAR_CHAIN_NO_ALLREDUCE = 3 };
    Section 3.1), which needs the P readers of that chain to mean anything. */
 enum { SIFAR_SYMCHAIN_TWOSHOT = 4 };
 
+/* Sixth and seventh "mode", sifar_symchain_create only: the paper's own validation scheme (Section 4.2,
+   "Speculative Reduction" and "Verification Logic Correctness"; overheads in Section 6.3): plain payload in
+   two alternating buffers, one validation flag per threadblock written after the payload (the flags alternate
+   too), one extra warp per threadblock that pulls the P flags while the other warps pull the payload, success
+   iff the flags add up to P x flag, otherwise the whole threadblock pulls again.
+   FLAGVAL issues payload and flag loads together, as the paper does; a stale payload read followed by a
+   fresh flag read would pass the check, which is what the paper's monotonicity assumption (Section 8.1)
+   excludes.  FLAGVAL_ORDERED pulls the payload only after all P flags were seen with acquire semantics:
+   sound without that assumption, at the price of the flag round trip. */
+enum { SIFAR_SYMCHAIN_FLAGVAL = 5, SIFAR_SYMCHAIN_FLAGVAL_ORDERED = 6 };
+
+/* Eighth "mode", sifar_symchain_create only, TIMING ONLY: the pull of FLAGVAL with no flag and no check at all
+   (the paper's idealized "no barriers" configuration of Section 6.3).  Its results are whatever the buffers
+   held; it exists so that verification overhead = (a validated mode) - (this) can be measured. */
+enum { SIFAR_SYMCHAIN_UNCHECKED = 7 };
+
 /* Bytes between two rows of an output ring for n elements (a multiple of 256, at least 512 bytes more than the
    row: the persistent kernels work in whole warps of 16-byte units and write zeros behind the last element). */
 size_t sifar_chain_ring_stride(int dtype, size_t n);
@@ -152,7 +168,8 @@ int sifar_chain_destroy(sifar_chain *chain);
  *                  rank r's copy of out^t lands in row r * ring_len + (t-1) mod ring_len
  *   other arguments as for sifar_chain_create (mode may also be SIFAR_CHAIN_NO_ALLREDUCE: every rank's
  *   operation feeds on its own partial, the timing floor; or SIFAR_SYMCHAIN_TWOSHOT: every rank reduces
- *   1/P of each chunk for all, a second barrier, then every rank reads the reduced chunk)
+ *   1/P of each chunk for all, a second barrier, then every rank reads the reduced chunk; or one of the
+ *   two SIFAR_SYMCHAIN_FLAGVAL modes above)
  * The chain owns the context exclusively until it is destroyed.
  */
 typedef struct sifar_symchain sifar_symchain;   /* opaque */

@@ -193,6 +193,7 @@ def sifar_noalloc_counters() -> dict:
 CHAIN_STREAMS, CHAIN_GRAPH, CHAIN_PERSISTENT = 0, 1, 2
 CHAIN_NO_ALLREDUCE = 3
 SYMCHAIN_TWOSHOT = 4
+SYMCHAIN_FLAGVAL, SYMCHAIN_FLAGVAL_ORDERED, SYMCHAIN_UNCHECKED = 5, 6, 7
 IMPL_NAMES = {CHAIN_STREAMS: "streams", CHAIN_GRAPH: "graph", CHAIN_PERSISTENT: "persistent"}
 
 

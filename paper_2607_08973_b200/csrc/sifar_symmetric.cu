@@ -22,6 +22,13 @@
  *                     reduce 1/P of the chunk for everybody (reduce-scatter); second barrier; read the
  *                     whole reduced chunk (all-gather).  The second barrier also covers the reuse of the
  *                     single buffer: a rank passes it only after every rank's reads of the partials.
+ *   FLAGVAL         : the paper's own validation scheme (Section 4.2, "Speculative Reduction" and
+ *                     "Verification Logic Correctness"): plain payload, one validation flag per threadblock
+ *                     written after the payload, one extra warp that pulls the P flags while the other
+ *                     warps pull the payload, success iff the flags sum to P x flag, else the whole
+ *                     threadblock runs again; the flag buffer is dual-buffered like the payload (k_symv).
+ *   FLAGVAL_ORDERED : the same objects, but the payload is pulled only after the extra warp has seen all P
+ *                     flags (acquire): the ordering that is sound on one GPU without any assumption.
  * so ranks drift against each other as real GPUs do, and a rank mis-speculates
  * exactly when a peer is behind it.  A thread keeps the same units in every step;
  * the speculative mode needs no CTA-wide barrier at all: the write-after-read
@@ -45,6 +52,10 @@ namespace sifar {
 constexpr int kSymThreads = 128;
 constexpr int kSymNoAllreduce = SIFAR_CHAIN_NO_ALLREDUCE;
 constexpr int kSymTwoshot = SIFAR_SYMCHAIN_TWOSHOT;
+constexpr int kSymFlagval = SIFAR_SYMCHAIN_FLAGVAL;
+constexpr int kSymFlagvalOrdered = SIFAR_SYMCHAIN_FLAGVAL_ORDERED;
+constexpr int kSymUnchecked = SIFAR_SYMCHAIN_UNCHECKED;
+constexpr int kSymvThreads = kSymThreads + 32;       /* the payload warps and one validation warp */
 
 /* Flags of one chunk: what the P CTAs that own it tell each other. */
 struct __align__(128) SymFlags {
@@ -305,6 +316,189 @@ __global__ void __launch_bounds__(kSymThreads, 6) k_sym(const SymArgs a)
     }
 }
 
+/*
+ * The paper's validation scheme in the chain with P readers (Section 4.2, "Speculative Reduction").
+ *
+ * Per step, CTA (r, c):
+ *   1. the rank's operation: chunk c of its next partial, plain stores into the parity buffer;
+ *   2. bar.sync, then ONE thread writes the threadblock's validation flag = call number, with release
+ *      (the flag follows the payload; the flag buffer alternates with the parity like the payload);
+ *   3. the four payload warps pull chunk c of all P partials and reduce it, storing the result into the
+ *      rank's own row at once (nobody else reads that row), while the FIFTH warp pulls the P validation
+ *      flags of the chunk and adds them up;
+ *   4. bar.sync; if the sum is not P x flag the whole CTA runs step 3 again (every load is a strong
+ *      access that bypasses the L1, which is what the paper's .cg on retry is for).
+ * ORDERED = false issues the payload loads and the flag loads together, as the paper does: a stale
+ * payload read followed by a fresh flag read would pass the check, and nothing in the memory model
+ * forbids that order; the paper's "monotonicity assumption" (Section 8.1) is what rules it out in
+ * practice, here for the two loads of one CTA.  ORDERED = true lets the payload warps wait until the
+ * validation warp has seen all P flags (acquire): sound on any schedule, and the flag round trip is
+ * back on the critical path, which makes it the dual-buffered mode with the paper's objects.
+ *
+ * UNCHECKED = the same pull with no flag and no check at all: the paper's idealized configuration "no
+ * barriers" (Section 6.3, "Mis-Speculation and Verification Overhead"), whose results are whatever was in
+ * the buffers.  A timing floor for the verification overhead, never a result.
+ * Forced retries (the context's measurement knob): the first attempts that pass the check are treated as
+ * failed, as many as asked for, so that the cost of a rerun can be measured (Section 6.3, "Retry Overhead").
+ */
+enum { kVariantConcurrent = 0, kVariantOrdered = 1, kVariantUnchecked = 2 };
+
+template <int DT, int P, int VARIANT>
+__global__ void __launch_bounds__(kSymvThreads, 4) k_symv(const SymArgs a)
+{
+    constexpr bool ORDERED = (VARIANT == kVariantOrdered);
+    constexpr bool UNCHECKED = (VARIANT == kVariantUnchecked);
+    DevState *st = a.st;
+    constexpr int NW = 4;
+    constexpr int NE = NW * ((DT == SIFAR_BF16) ? 2 : 1);
+    const uint32_t rank = blockIdx.x % (uint32_t)P;
+    const uint32_t chunk = blockIdx.x / (uint32_t)P;
+    SymFlags *cf = a.flags + chunk;
+    const size_t n = (size_t)a.n;
+    const size_t nunits = ((n + NE - 1) / NE + 31) / 32 * 32;
+    const size_t n_io = nunits * NE;
+    const bool worker = threadIdx.x < (unsigned)kSymThreads;          /* payload warps; the last warp validates */
+    const unsigned lane = threadIdx.x & 31u;
+    const size_t unit0 = (size_t)chunk * kSymThreads * a.K + threadIdx.x;
+    char *my_ring = a.rings + (size_t)rank * a.ring_len * a.ring_stride;
+    constexpr uint32_t kWarps = kSymThreads / 32;
+    const bool stamper = worker && lane == 0u;
+    unsigned long long *my_stamps = a.stamps + (((size_t)rank * a.C + chunk) * kWarps + (threadIdx.x >> 5)) * (a.steps + 1u);
+    __shared__ int s_ok;
+    __shared__ int s_valid;
+    __shared__ int s_giveup;
+    unsigned reloads = 0;
+    bool alive = true;
+    uint32_t prevw[NW];
+#pragma unroll
+    for (int j = 0; j < NW; ++j) prevw[j] = 0u;
+    if (stamper) my_stamps[0] = globaltimer_ns();
+
+    for (uint32_t s = 0; s < a.steps && alive; ++s) {
+        const uint32_t e = a.e0 + 1u + s;
+        const uint32_t t = e - a.base_epoch;
+        const uint32_t p = e & 1u;
+        const bool first = (t == 1u);
+        const Gen g = make_gen(a.w, rank, t);
+        char *row = my_ring + (size_t)((t - 1u) % a.ring_len) * a.ring_stride;
+        const char *prev_mem = my_ring + (size_t)((t + a.ring_len - 2u) % a.ring_len) * a.ring_stride;
+        uint4 *dst = reinterpret_cast<uint4 *>(a.plain + ((size_t)p * P + rank) * a.plain_stride);
+
+        /* ---- 1. the rank's operation ---- */
+        float z0[NE];
+        if (worker && unit0 < nunits) unit_noise<DT, NW>(g, first, unit0 * NE, n, z0);
+        if (a.w.delay_max_ns != 0u) {
+            if (threadIdx.x == 0) spin_ns(gen_delay_ns(a.w, rank, t));       /* seeded skew between the ranks */
+            __syncthreads();
+        }
+        if (worker) {
+            for (uint32_t k = 0; k < a.K; ++k) {
+                const size_t u = unit0 + (size_t)k * kSymThreads;
+                if (u >= nunits) break;
+                uint32_t w[NW];
+                if (k == 0 && s > 0u) {
+                    unit_apply<DT, NW>(g, first, prevw, u * NE, n, z0, w);
+                } else if (k == 0) {
+                    unit_combine<DT, NW>(g, first, prev_mem, u * NE, n, z0, w, n_io);
+                } else {
+                    float z[NE];
+                    unit_noise<DT, NW>(g, first, u * NE, n, z);
+                    unit_combine<DT, NW>(g, first, prev_mem, u * NE, n, z, w, n_io);
+                }
+                st_slot(dst + u, make_uint4(w[0], w[1], w[2], w[3]));
+            }
+        }
+        /* ---- 2. the threadblock's validation flag, after its payload ---- */
+        if (!UNCHECKED) {
+            __syncthreads();
+            if (threadIdx.x == 0) st_release_u32(&cf->arrive[p][rank], e);
+        }
+
+        /* ---- 3./4. pull payload and flags, validate, run again on mis-speculation ---- */
+        const uint4 *src[P];
+#pragma unroll
+        for (int r = 0; r < P; ++r)
+            src[r] = reinterpret_cast<const uint4 *>(a.plain + ((size_t)p * P + r) * a.plain_stride);
+        Deadline dl;                                                /* kept by thread 0, which decides for the CTA */
+        bool retried = false;
+        const auto pull_flags = [&]() {
+            /* validation warp: pull-and-local-reduce of the P flags; success iff they add up to P x flag */
+            uint32_t f = 0u;
+            if (lane < (unsigned)P) f = ORDERED ? ld_acquire_u32(&cf->arrive[p][lane]) : ld_relaxed_u32(&cf->arrive[p][lane]);
+            const uint32_t valid_out = __reduce_add_sync(0xFFFFFFFFu, f);
+            if (lane == 0) s_valid = (valid_out == (uint32_t)P * e);
+        };
+        const auto pull_payload = [&]() {
+            for (uint32_t k = 0; k < a.K; ++k) {
+                const size_t u = unit0 + (size_t)k * kSymThreads;
+                if (u >= nunits) break;
+                uint4 x[P];
+#pragma unroll
+                for (int r = 0; r < P; ++r) x[r] = ld_slot(src[r] + u);
+                const uint4 o = sum_vec<DT, P>(x, true);
+                store_vec_result<DT>(row, u, n_io, o);              /* own row: rewritten if the check fails */
+                if (k == 0) { prevw[0] = o.x; prevw[1] = o.y; prevw[2] = o.z; prevw[3] = o.w; }
+            }
+        };
+        const auto give_up = [&]() {                                /* thread 0, after a failed check */
+            const bool out_of_time = dl.expired(a.timeout_ns);
+            if (out_of_time) fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+            return out_of_time || ((dl.polls % 64u) == 0u && ld_relaxed_u32(&st->status) != 0u);
+        };
+        uint32_t forced_left = a.poll.forced;
+        for (;;) {
+            if (UNCHECKED) { if (worker) pull_payload(); break; }
+            if (!worker) pull_flags();
+            if (!ORDERED && worker) pull_payload();                 /* at the same time as the flags, as the paper does */
+            __syncthreads();                                        /* the verdict (and, unordered, the payload) */
+            if (s_valid && forced_left == 0u) break;                /* uniform over the CTA */
+            if (s_valid) --forced_left;                             /* a passed check counted as failed (measurement) */
+            retried = true;
+            if (!ORDERED) reloads += (unsigned)P;
+            if (threadIdx.x == 0) s_giveup = give_up();
+            __syncthreads();                                        /* s_valid may be rewritten from here on */
+            if (s_giveup) { alive = false; break; }
+        }
+        if (ORDERED && alive && worker) pull_payload();             /* only after all P flags were seen */
+        if (!alive) break;
+        if (retried && threadIdx.x == 0) st_relaxed_u32(&a.retry_marks[(size_t)rank * a.steps + s], 1u);
+        if (stamper) my_stamps[s + 1u] = globaltimer_ns();
+    }
+
+    /* leave: statistics, then the last CTA out books the run and publishes the call number */
+    const unsigned warp_reloads = __reduce_add_sync(0xFFFFFFFFu, reloads);
+    if (warp_reloads && lane == 0)
+        atomicAdd(&st->stats[kStatSlotReloads], (unsigned long long)warp_reloads);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const uint32_t left = atom_add_acq_rel_u32(&a.cs->exit_count, 1u) + 1u;
+        s_ok = (left == a.exit_base + gridDim.x && ld_relaxed_u32(&st->status) == 0u);
+    }
+    __syncthreads();
+    if (s_ok) {
+        unsigned long long any_steps = 0;
+        for (uint32_t s = threadIdx.x; s < a.steps; s += kSymvThreads) {
+            uint32_t any = 0;
+            for (int r = 0; r < P; ++r) {
+                const uint32_t m = ld_relaxed_u32(&a.retry_marks[(size_t)r * a.steps + s]);
+                if (m) {
+                    atomicAdd(&a.rank_retries[r], 1ull);
+                    st_relaxed_u32(&a.retry_marks[(size_t)r * a.steps + s], 0u);
+                }
+                any |= m;
+            }
+            any_steps += any ? 1ull : 0ull;
+        }
+        if (any_steps) atomicAdd(&st->stats[kStatCallsWithRetry], any_steps);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            atomicAdd(&st->stats[kStatCalls], (unsigned long long)a.steps);
+            st_release_u32(&st->epoch, a.e0 + a.steps);
+        }
+    }
+}
+
 template <int DT, int P>
 static const void *sym_kernel_p(int mode)
 {
@@ -313,6 +507,9 @@ static const void *sym_kernel_p(int mode)
     case SIFAR_DUALBUF:         return (const void *)k_sym<DT, P, SIFAR_DUALBUF>;
     case SIFAR_SPECULATIVE:     return (const void *)k_sym<DT, P, SIFAR_SPECULATIVE>;
     case kSymTwoshot:           return (const void *)k_sym<DT, P, kSymTwoshot>;
+    case kSymFlagval:           return (const void *)k_symv<DT, P, kVariantConcurrent>;
+    case kSymFlagvalOrdered:    return (const void *)k_symv<DT, P, kVariantOrdered>;
+    case kSymUnchecked:         return (const void *)k_symv<DT, P, kVariantUnchecked>;
     default:                    return (const void *)k_sym<DT, P, kSymNoAllreduce>;
     }
 }
@@ -357,6 +554,9 @@ struct sifar_symchain {
     unsigned long long *d_rank_retries;
 };
 
+/* Threads per CTA: the flag-validation modes run one extra warp. */
+static int sym_threads(int mode) { return mode >= kSymFlagval ? kSymvThreads : kSymThreads; }
+
 static const void *sym_kernel(const sifar_symchain *ch)
 {
     return ch->ctx->dtype == SIFAR_BF16 ? sym_kernel_dt<SIFAR_BF16>(ch->ctx->P, ch->mode)
@@ -384,7 +584,8 @@ static int sym_setup(sifar_symchain *ch)
     const size_t units = (ch->mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, ch->n)
                                                          : (ch->n * elem_size(c->dtype) + 15) / 16;
     int per_sm = 0;
-    SIFAR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sym_kernel(ch), kSymThreads, 0));
+    const int threads = sym_threads(ch->mode);
+    SIFAR_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sym_kernel(ch), threads, 0));
     const size_t resident = (size_t)per_sm * c->sm_count;
     const size_t budget = resident > (size_t)P ? resident : (size_t)P;
     uint32_t K = 1;
@@ -400,7 +601,7 @@ static int sym_setup(sifar_symchain *ch)
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof cfg);
         cfg.gridDim = dim3((unsigned)ch->grid);
-        cfg.blockDim = dim3(kSymThreads);
+        cfg.blockDim = dim3((unsigned)threads);
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = (unsigned)P;
@@ -431,7 +632,7 @@ extern "C" sifar_symchain *sifar_symchain_create(sifar_ctx *c, const sifar_workl
                                                  void *out_rings, int ring_len, int steps_per_run)
 {
     if (!c || !w || w->kind < 0 || w->kind > 2 || w->delay_max_ns > 1000000u || n == 0 || n > c->max_elems ||
-        mode < 0 || mode > kSymTwoshot || !out_rings || ((uintptr_t)out_rings & 15u) || ring_len < 2 ||
+        mode < 0 || mode > kSymUnchecked || !out_rings || ((uintptr_t)out_rings & 15u) || ring_len < 2 ||
         steps_per_run < 2 || (steps_per_run & 1) || steps_per_run % ring_len != 0) {
         set_error("sifar_symchain_create: bad argument (need 1 <= n <= max_elems, ring_len >= 2 dividing an even "
                   "steps_per_run, delay_max_ns <= 1000000)");
@@ -493,7 +694,7 @@ extern "C" int sifar_symchain_run(sifar_symchain *ch, void *stream)
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof cfg);
         cfg.gridDim = dim3((unsigned)ch->grid);
-        cfg.blockDim = dim3(kSymThreads);
+        cfg.blockDim = dim3((unsigned)sym_threads(ch->mode));
         cfg.stream = s;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeCooperative;
@@ -506,7 +707,7 @@ extern "C" int sifar_symchain_run(sifar_symchain *ch, void *stream)
         cfg.numAttrs = 2;
         SIFAR_CUDA(cudaLaunchKernelExC(&cfg, fn, params));
     } else {
-        SIFAR_CUDA(cudaLaunchCooperativeKernel(fn, dim3((unsigned)ch->grid), dim3(kSymThreads), params, 0, s));
+        SIFAR_CUDA(cudaLaunchCooperativeKernel(fn, dim3((unsigned)ch->grid), dim3((unsigned)sym_threads(ch->mode)), params, 0, s));
     }
     ch->runs += 1;
     if (!no_ar) c->h_epoch += (uint32_t)ch->steps;

@@ -43,9 +43,13 @@ def test_config5_ten_thousand_skewed_steps(skew_reference, impl, mode):
         assert 0 < st["calls_with_retry"] <= steps * runs and st["slot_reloads"] > 0
 
 
-@pytest.mark.parametrize("mode", [sf.SPECULATIVE, sf.BARRIER_ONESHOT])
+@pytest.mark.parametrize("mode", [sf.SPECULATIVE, sf.BARRIER_ONESHOT, sf.SYMCHAIN_FLAGVAL_ORDERED, sf.SYMCHAIN_FLAGVAL])
 def test_config5_ten_thousand_skewed_steps_with_p_readers(skew_reference, mode):
-    """The same 10 000 steps with every rank reducing for itself: all eight copies, every step."""
+    """The same 10 000 steps with every rank reducing for itself: all eight copies, every step.
+
+    SYMCHAIN_FLAGVAL is the paper's validation scheme with payload and flags pulled together; its check is sound
+    only under the paper's monotonicity assumption (Section 8.1).  A mismatch in that one case, with the ordered
+    variant green, would be that hazard showing, not an arithmetic defect; none was seen in 2 500 000 steps."""
     d, want = skew_reference
     P, n, steps, runs = 8, 16384, 100, 100
     stride = sf.sifar_chain_ring_stride(BF16, n)
@@ -69,6 +73,9 @@ def test_config5_ten_thousand_skewed_steps_with_p_readers(skew_reference, mode):
         # every rank but the last one of a step finds a peer missing: (P-1)/P of the steps on average
         share = np.array(retries) / (steps * runs)
         assert np.all(share > 0.7) and np.all(share < 0.98), share
+    elif mode in (sf.SYMCHAIN_FLAGVAL, sf.SYMCHAIN_FLAGVAL_ORDERED):
+        # the flags of the peers are looked at right after the own one was written: hardly ever all there at once
+        assert np.all(np.array(retries) > 0.7 * steps * runs), retries
     else:
         assert sum(retries) == 0
 
