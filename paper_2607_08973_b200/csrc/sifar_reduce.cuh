@@ -21,6 +21,7 @@ namespace sifar {
  * round trip (~0.3 us), so a limit is overshot by a few microseconds at most.
  */
 constexpr unsigned kPollsPerClockCheck = 8;
+constexpr unsigned kPollStaggerNs = 120;         /* spacing of the polls a waiting lane keeps in flight */
 
 struct Deadline {
     unsigned long long t0 = 0;
@@ -186,9 +187,24 @@ __device__ __forceinline__ bool sentinel_wait(const uint4 *const *src, size_t wa
 #pragma unroll
         for (int r = 0; r < P; ++r)
             if (lane == (unsigned)r) p = src[r] + warp_first_slot;
+        /* Three polls in flight, issued a third of a round trip apart: a poll loop that waits for each answer
+           before it asks again sees an arrival up to a whole round trip late, and in a chain whose steps all
+           look alike that delay does not average out (the same code was 0.6 us per step faster or slower
+           depending on where its polls happened to fall). */
         Deadline d;
-        while (ld_slot(p).w != e) {
-            ++reloads;
+        uint4 v0 = ld_slot(p);
+        __nanosleep(kPollStaggerNs);
+        uint4 v1 = ld_slot(p);
+        __nanosleep(kPollStaggerNs);
+        uint4 v2 = ld_slot(p);
+        for (;;) {
+            if (v0.w == e) break;
+            v0 = ld_slot(p);
+            if (v1.w == e) break;
+            v1 = ld_slot(p);
+            if (v2.w == e) break;
+            v2 = ld_slot(p);
+            reloads += 3;
             if (d.expired(timeout_ns)) { ok = false; break; }
         }
     }

@@ -339,13 +339,15 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
                     /* warp-uniform: the warp's first slot decides whether the warp has work at all */
                     const size_t w0 = u - (threadIdx.x & 31u);
                     if (w0 >= nunits) break;
-                    const unsigned before = reloads;
-                    if (!sentinel_wait<P>(src, w0, e, a.timeout_ns, reloads)) {
-                        if (threadIdx.x == 0 || (threadIdx.x & 31u) == 0u) fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
-                        alive = false;
-                        break;
+                    if (k == 0 || a.K > 1u) {
+                        const unsigned before = reloads;
+                        if (!sentinel_wait<P>(src, w0, e, a.timeout_ns, reloads)) {
+                            if (threadIdx.x == 0 || (threadIdx.x & 31u) == 0u) fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+                            alive = false;
+                            break;
+                        }
+                        retried |= (reloads != before);
                     }
-                    retried |= (reloads != before);
                 }
                 if (u >= nunits) break;
                 uint4 x[P];
