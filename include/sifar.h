@@ -241,10 +241,13 @@ int sifar_debug_set_epoch(sifar_ctx *ctx, unsigned calls_so_far);
  * The paper has no counterpart: it targets decode payloads of 8-32 KB (Section 5),
  * where the tags of the slots cost nothing that matters.  For large payloads the
  * tagged slots move a third more bytes than plain data, which is what bounds the
- * reducer there, so from 16 MiB for all P partials together the speculative mode
+ * reducer there, so from 8 MiB for all P partials together the speculative mode
  * keeps the early start (Section 3.5) but validates per block instead of per slot:
  *
- * SIFAR_FORMAT_SLOTS   16-byte slots {12 data bytes, 4-byte tag}; no flag at all.
+ * SIFAR_FORMAT_SLOTS   16-byte slots {12 data bytes, 4-byte tag}; no flag at all.  (A library built with
+ *                      -DSIFAR_SLOT_S8X2, libsifar_s8x2.so, uses two halves {4 data bytes, tag} per slot
+ *                      instead, each valid on its own: it needs only 64-bit atomicity and is the fallback
+ *                      should a 16-byte access ever be seen torn; sifar_slot_count() tells the geometry.)
  * SIFAR_FORMAT_TILES   plain elements at the start of the same rank buffer, plus one
  *                      arrival flag per block of 16 KiB (8192 bf16 / 4096 fp32
  *                      elements; the last block may be short), set to the call number

@@ -113,12 +113,59 @@ __device__ __forceinline__ unsigned long long globaltimer_ns()
     return t;
 }
 
-/* One tagged slot: three data words and the call number, in one 16-byte store. */
+/*
+ * Slot format.  Default ("S12"): {w0, w1, w2, tag}, written and read with one 16-byte access; a slot counts
+ * iff its tag is the call number.  Fallback, compiled with -DSIFAR_SLOT_S8X2: two halves {w0, tag} and
+ * {w1, tag}, each written with one 8-byte store and valid on its own, so that only 64-bit single-copy
+ * atomicity is relied on (the memory model's scalar guarantee); 8 data bytes per 16-byte slot instead of 12.
+ * Should the 16-byte check (sifar_tear_check) ever report a torn slot, this is the layout to build.
+ */
+#ifdef SIFAR_SLOT_S8X2
+constexpr int kSlotDataWords = 2;
+#else
+constexpr int kSlotDataWords = 3;
+#endif
+
+/* Does the slot image carry call number `tag` (in the fallback format: both of its halves)? */
+__device__ __forceinline__ bool slot_valid(const uint4 &v, uint32_t tag)
+{
+#ifdef SIFAR_SLOT_S8X2
+    return v.y == tag && v.w == tag;
+#else
+    return v.w == tag;
+#endif
+}
+
+/* Data word j (0 .. kSlotDataWords - 1) of a slot image. */
+__device__ __forceinline__ uint32_t slot_word(const uint4 &v, int j)
+{
+#ifdef SIFAR_SLOT_S8X2
+    return j == 0 ? v.x : v.z;
+#else
+    return j == 0 ? v.x : j == 1 ? v.y : v.z;
+#endif
+}
+
+/* One tagged slot: kSlotDataWords data words and the call number. */
+__device__ __forceinline__ void store_slot_words(uint4 *slots, size_t i, const uint32_t (&w)[kSlotDataWords], uint32_t tag)
+{
+#ifdef SIFAR_SLOT_S8X2
+    uint32_t *p = reinterpret_cast<uint32_t *>(slots + i);
+    asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" :: "l"(p), "r"(w[0]), "r"(tag) : "memory");
+    asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" :: "l"(p + 2), "r"(w[1]), "r"(tag) : "memory");
+#else
+    st_slot(slots + i, make_uint4(w[0], w[1], w[2], tag));
+#endif
+}
+
+#ifndef SIFAR_SLOT_S8X2
+/* The default format spelled out: three data words and the call number, in one 16-byte store. */
 __device__ __forceinline__ void store_slot(uint4 *slots, size_t i, uint32_t w0, uint32_t w1,
                                            uint32_t w2, uint32_t tag)
 {
     st_slot(slots + i, make_uint4(w0, w1, w2, tag));
 }
+#endif
 
 /*
  * Arrival of one rank in the barrier modes.  Every thread of every CTA that

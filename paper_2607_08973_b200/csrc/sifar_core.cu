@@ -202,7 +202,7 @@ __device__ __forceinline__ bool tile_spec(const ReduceArgs &a, size_t tile, size
         for (int r = 0; r < P; ++r) x[r] = ld_slot(a.src[r] + s);
         /* validation (Section 4.2): a slot counts iff it carries this call's tag; stale ones are re-loaded */
         if (!validate_slot<P>(x, a.src, s, e, limit_ns, a.poll, reloads)) { ok = false; continue; }
-        store_slot_result<DT>(a.out, s, (size_t)a.n, sum_vec<DT, P>(x, false));
+        store_slot_result<DT>(a.out, s, (size_t)a.n, sum_slot<DT, P>(x));
     }
     return ok;
 }
@@ -523,7 +523,7 @@ template <int DT, int P>
 __global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
 {
     constexpr int U = Unroll<P>::value;
-    constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;
+    constexpr int EPS = kSlotDataWords * ((DT == SIFAR_BF16) ? 2 : 1);
     DevState *st = a.st;
     const size_t nslots = ((size_t)a.n + EPS - 1) / EPS;
     const size_t tile = blockIdx.x;
@@ -575,7 +575,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_spec(const ReduceArgs a)
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const size_t s = base + (size_t)u * kThreads;
-                if (s < nslots) store_slot_result<DT>(a.out, s, (size_t)a.n, sum_vec<DT, P>(x[u], false));
+                if (s < nslots) store_slot_result<DT>(a.out, s, (size_t)a.n, sum_slot<DT, P>(x[u]));
             }
         } else if (!a.two_phase) {
             fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
@@ -690,7 +690,8 @@ __device__ __forceinline__ void pack_body(const PackArgs &a)
         }
         signal_arrival(&st->pack_count[a.rank], gridDim.x, &st->arrive[e & 1u][a.rank], e);
     } else {
-        constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;
+        constexpr int EPS = kSlotDataWords * ((DT == SIFAR_BF16) ? 2 : 1);
+        constexpr int NW = kSlotDataWords;
         const size_t nslots = ((size_t)a.n + EPS - 1) / EPS;
         uint4 *slots = reinterpret_cast<uint4 *>(a.dst);
         const uint32_t *src32 = reinterpret_cast<const uint32_t *>(a.src);
@@ -698,20 +699,24 @@ __device__ __forceinline__ void pack_body(const PackArgs &a)
         const size_t nfull = (size_t)a.n / EPS;
         size_t s = tid;
         for (; s + (kPackUnroll - 1) * nthreads < nfull; s += kPackUnroll * nthreads) {
-            uint32_t w[kPackUnroll][3];
+            uint32_t w[kPackUnroll][NW];
 #pragma unroll
             for (int j = 0; j < kPackUnroll; ++j) {
-                const uint32_t *p = src32 + (s + j * nthreads) * 3;
-                w[j][0] = __ldcs(p); w[j][1] = __ldcs(p + 1); w[j][2] = __ldcs(p + 2);
+                const uint32_t *p = src32 + (s + j * nthreads) * NW;
+#pragma unroll
+                for (int q = 0; q < NW; ++q) w[j][q] = __ldcs(p + q);
             }
 #pragma unroll
-            for (int j = 0; j < kPackUnroll; ++j) store_slot(slots, s + j * nthreads, w[j][0], w[j][1], w[j][2], e);
+            for (int j = 0; j < kPackUnroll; ++j) store_slot_words(slots, s + j * nthreads, w[j], e);
         }
         for (; s < nslots; s += nthreads) {
-            uint32_t w[3] = {0u, 0u, 0u};
+            uint32_t w[NW];
+#pragma unroll
+            for (int q = 0; q < NW; ++q) w[q] = 0u;
             const size_t i0 = s * EPS;
             if (i0 + EPS <= a.n) {
-                w[0] = src32[s * 3]; w[1] = src32[s * 3 + 1]; w[2] = src32[s * 3 + 2];
+#pragma unroll
+                for (int q = 0; q < NW; ++q) w[q] = src32[s * NW + q];
             } else if (DT == SIFAR_BF16) {
                 const uint16_t *src16 = reinterpret_cast<const uint16_t *>(a.src);
                 for (int k = 0; k < EPS && i0 + k < a.n; ++k)
@@ -719,7 +724,7 @@ __device__ __forceinline__ void pack_body(const PackArgs &a)
             } else {
                 for (int k = 0; k < EPS && i0 + k < a.n; ++k) w[k] = src32[i0 + k];
             }
-            store_slot(slots, s, w[0], w[1], w[2], e);
+            store_slot_words(slots, s, w, e);
         }
     }
 }
@@ -883,12 +888,13 @@ size_t sifar::reduce_tiles(const sifar_ctx *ctx, size_t n, int mode)
 
 /*
  * Format of the speculative mode by size.  Slots carry their own tags (no flag, no dependent round trip)
- * but move a third more bytes; from 16 MiB for all P partials together, where bandwidth is what counts,
+ * but move a third more bytes; from 8 MiB for all P partials together (1 MiB per rank at P = 8: where the plain
+ * reducer overtakes the slot reducer on ready data on B200), where bandwidth is what counts,
  * the partial travels as plain data with one arrival flag per 16 KiB block.
  */
 static int spec_format(int P, int dtype, size_t n)
 {
-    constexpr size_t kTilesFromBytes = (size_t)16 << 20;
+    constexpr size_t kTilesFromBytes = (size_t)8 << 20;
     return (size_t)P * n * sifar::elem_size(dtype) < kTilesFromBytes ? SIFAR_FORMAT_SLOTS : SIFAR_FORMAT_TILES;
 }
 

@@ -61,7 +61,7 @@ __device__ __forceinline__ void fail(DevState *st, volatile int *host_status, in
 
 /* Element geometry */
 __host__ __device__ inline size_t elem_size(int dtype) { return dtype == SIFAR_BF16 ? 2 : 4; }
-__host__ __device__ inline size_t elems_per_slot(int dtype) { return dtype == SIFAR_BF16 ? 6 : 3; }
+__host__ __device__ inline size_t elems_per_slot(int dtype) { return (size_t)kSlotDataWords * (dtype == SIFAR_BF16 ? 2 : 1); }
 __host__ __device__ inline size_t slots_for(int dtype, size_t n)
 {
     size_t k = elems_per_slot(dtype);

@@ -107,6 +107,21 @@ __device__ __forceinline__ uint4 sum_vec(const uint4 (&x)[P], bool with_w)
     return o;
 }
 
+/* The data words of P slot images, summed in rank order: word j of the result in .x, .y (, .z). */
+template <int DT, int P>
+__device__ __forceinline__ uint4 sum_slot(const uint4 (&x)[P])
+{
+    uint32_t o[3] = {0u, 0u, 0u};
+#pragma unroll
+    for (int j = 0; j < kSlotDataWords; ++j) {
+        uint32_t a[P];
+#pragma unroll
+        for (int r = 0; r < P; ++r) a[r] = slot_word(x[r], j);
+        o[j] = sum_word<DT, P>(a);
+    }
+    return make_uint4(o[0], o[1], o[2], 0u);
+}
+
 /* Vectors (plain) or slots (speculative) a thread keeps in flight per rank. */
 template <int P> struct Unroll { static constexpr int value = (P <= 2) ? 4 : (P <= 4) ? 2 : 1; };
 
@@ -147,7 +162,7 @@ __device__ __forceinline__ bool revalidate(uint4 (&x)[P], uint32_t stale, const 
         const uint32_t before = stale;
 #pragma unroll
         for (int r = 0; r < P; ++r)
-            if ((pending & (1u << r)) && x[r].w == e) stale &= ~(1u << r);
+            if ((pending & (1u << r)) && slot_valid(x[r], e)) stale &= ~(1u << r);
         reloads += __popc(pending);
         if (!WIDE) burst = !burst && stale != before;    /* the polled rank arrived: look at all others once */
         if (round_stamps && round < 8u) round_stamps[round] = globaltimer_ns();
@@ -198,11 +213,11 @@ __device__ __forceinline__ bool sentinel_wait(const uint4 *const *src, size_t wa
         __nanosleep(kPollStaggerNs);
         uint4 v2 = ld_slot(p);
         for (;;) {
-            if (v0.w == e) break;
+            if (slot_valid(v0, e)) break;
             v0 = ld_slot(p);
-            if (v1.w == e) break;
+            if (slot_valid(v1, e)) break;
             v1 = ld_slot(p);
-            if (v2.w == e) break;
+            if (slot_valid(v2, e)) break;
             v2 = ld_slot(p);
             reloads += 3;
             if (d.expired(timeout_ns)) { ok = false; break; }
@@ -218,7 +233,7 @@ __device__ __forceinline__ bool validate_once(uint4 (&x)[P], const uint4 *const 
 {
     uint32_t stale = 0;
 #pragma unroll
-    for (int r = 0; r < P; ++r) stale |= (uint32_t)(x[r].w != e) << r;
+    for (int r = 0; r < P; ++r) stale |= (uint32_t)(!slot_valid(x[r], e)) << r;
     if (stale == 0u) return true;
     return shape.wide ? revalidate<P, true>(x, stale, src, s, e, timeout_ns, shape.pace_ns, reloads, round_stamps)
                       : revalidate<P, false>(x, stale, src, s, e, timeout_ns, shape.pace_ns, reloads, round_stamps);
@@ -251,15 +266,16 @@ __device__ __forceinline__ bool validate_slot(uint4 (&x)[P], const uint4 *const 
 /* ------------------------------------------------------------------------ */
 /* result stores                                                             */
 /* ------------------------------------------------------------------------ */
-/* The 12 data bytes of reduced slot s go to elements [s*EPS, s*EPS+EPS) of out; a short last slot is masked. */
+/* The data bytes of reduced slot s go to elements [s*EPS, s*EPS+EPS) of out; a short last slot is masked. */
 template <int DT>
 __device__ __forceinline__ void store_slot_result(void *out, size_t s, size_t n, const uint4 &o)
 {
-    constexpr int EPS = (DT == SIFAR_BF16) ? 6 : 3;
+    constexpr int EPS = kSlotDataWords * ((DT == SIFAR_BF16) ? 2 : 1);
     const size_t i0 = s * EPS;
     if (i0 + EPS <= n) {
-        uint32_t *dst = reinterpret_cast<uint32_t *>(out) + s * 3;
-        dst[0] = o.x; dst[1] = o.y; dst[2] = o.z;
+        uint32_t *dst = reinterpret_cast<uint32_t *>(out) + s * kSlotDataWords;
+        dst[0] = o.x; dst[1] = o.y;
+        if (kSlotDataWords == 3) dst[2] = o.z;
     } else if (DT == SIFAR_BF16) {
         uint16_t *dst = reinterpret_cast<uint16_t *>(out) + i0;
         const uint32_t w[3] = {o.x, o.y, o.z};

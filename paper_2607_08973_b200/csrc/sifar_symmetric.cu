@@ -43,6 +43,9 @@
 #include <vector>
 
 #include "sifar_internal.cuh"
+#ifdef SIFAR_SLOT_S8X2
+#error "the decode-step chains are written for the default slot format; the fallback format is built for libsifar only"
+#endif
 #include "sifar_reduce.cuh"
 #include "sifar_gen.cuh"
 #include "sifar_workload.h"

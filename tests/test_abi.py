@@ -49,14 +49,14 @@ def test_geometry_helpers_need_no_gpu():
 def test_speculative_format_choice_needs_no_gpu():
     import pytest
     from paper_2607_08973_b200 import binding as sf
-    # tagged slots while all P partials together stay below 16 MiB, flagged tiles of plain data from there on
+    # tagged slots while all P partials together stay below 8 MiB, flagged tiles of plain data from there on
     assert sf.sifar_spec_format(8, sf.BF16, 4096) == sf.FORMAT_SLOTS
-    assert sf.sifar_spec_format(8, sf.BF16, (1 << 20) - 1) == sf.FORMAT_SLOTS
-    assert sf.sifar_spec_format(8, sf.BF16, 1 << 20) == sf.FORMAT_TILES            # 8 x 2 MiB
-    assert sf.sifar_spec_format(2, sf.BF16, (1 << 22) - 1) == sf.FORMAT_SLOTS
-    assert sf.sifar_spec_format(2, sf.BF16, 1 << 22) == sf.FORMAT_TILES            # 2 x 8 MiB
-    assert sf.sifar_spec_format(8, sf.F32, (1 << 19) - 1) == sf.FORMAT_SLOTS
-    assert sf.sifar_spec_format(8, sf.F32, 1 << 19) == sf.FORMAT_TILES
+    assert sf.sifar_spec_format(8, sf.BF16, (1 << 19) - 1) == sf.FORMAT_SLOTS
+    assert sf.sifar_spec_format(8, sf.BF16, 1 << 19) == sf.FORMAT_TILES            # 8 x 1 MiB
+    assert sf.sifar_spec_format(2, sf.BF16, (1 << 21) - 1) == sf.FORMAT_SLOTS
+    assert sf.sifar_spec_format(2, sf.BF16, 1 << 21) == sf.FORMAT_TILES            # 2 x 4 MiB
+    assert sf.sifar_spec_format(8, sf.F32, (1 << 18) - 1) == sf.FORMAT_SLOTS
+    assert sf.sifar_spec_format(8, sf.F32, 1 << 18) == sf.FORMAT_TILES
     assert sf.sifar_spec_format(1, sf.BF16, 0) == sf.FORMAT_SLOTS
     for bad in ((0, sf.BF16, 1), (9, sf.BF16, 1), (2, 7, 1)):
         with pytest.raises(sf.SifarError):

@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 
 def _first_tiles_n(P, dtype, extra):
     """Smallest n in the flagged-tile format, plus `extra` elements."""
-    n = (16 << 20) // (P * (2 if dtype == BF16 else 4)) + extra
+    n = (8 << 20) // (P * (2 if dtype == BF16 else 4)) + extra
     assert sf.sifar_spec_format(P, dtype, n) == sf.FORMAT_TILES
     return n
 
