@@ -88,6 +88,7 @@ struct ReduceArgs {
     uint32_t flag_shift;
     uint32_t early;          /* 1: reads do not wait for the stream's previous kernel, writes do     */
     uint32_t e_host;         /* the call number the host expects, or 0: take it from device memory   */
+    uint32_t pdl;            /* host side only: launch with programmatic stream serialization         */
 };
 
 struct PackArgs {
@@ -825,9 +826,10 @@ static cudaError_t launch_k(K kernel, int grid, cudaStream_t s, const ReduceArgs
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
-    /* only for grids above the SM count: at decode payloads the early-resident reducer measurably slows
-       the graph chains and the host path (its blocked CTAs sit beside the kernels it waits for) */
-    cfg.attrs = at; cfg.numAttrs = (g_pdl && a.two_phase) ? 1 : 0;
+    /* for grids above the SM count, and for any grid whose producers are known to run on other streams: at
+       decode payloads a reducer that becomes resident early beside the very kernels it waits for measurably
+       slows the graph chains and the host path */
+    cfg.attrs = at; cfg.numAttrs = (g_pdl && (a.two_phase || a.pdl)) ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, a);
 }
 
@@ -953,7 +955,8 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
         else cudaGetLastError();
     }
     /* Early reads need programmatic launch to mean anything, and the baseline keeps the plain stream order. */
-    a.early = (rl.early && g_pdl && a.two_phase && rl.mode != SIFAR_BARRIER_ONESHOT && !rl.programmatic_event) ? 1u : 0u;
+    a.pdl = (rl.early && g_pdl && !rl.programmatic_event) ? 1u : 0u;
+    a.early = (a.pdl && rl.mode != SIFAR_BARRIER_ONESHOT) ? 1u : 0u;
     g_programmatic_event = rl.programmatic_event;
     cudaError_t err = (ctx->dtype == SIFAR_BF16)
         ? launch_reduce_dt<SIFAR_BF16>(ctx->P, kernel_mode, (int)ntiles, stream, a)

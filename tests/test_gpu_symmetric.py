@@ -138,7 +138,7 @@ def test_bad_arguments_are_refused():
         L = sf._wl()
         for args in ((ctx.h, ctypes.byref(w), 0, 2, rings.data_ptr(), 4, 4),
                      (ctx.h, ctypes.byref(w), 65, 2, rings.data_ptr(), 4, 4),
-                     (ctx.h, ctypes.byref(w), 64, 5, rings.data_ptr(), 4, 4),
+                     (ctx.h, ctypes.byref(w), 64, 8, rings.data_ptr(), 4, 4),
                      (ctx.h, ctypes.byref(w), 64, 2, None, 4, 4),
                      (ctx.h, ctypes.byref(w), 64, 2, rings.data_ptr(), 1, 4),
                      (ctx.h, ctypes.byref(w), 64, 2, rings.data_ptr(), 4, 6),
