@@ -31,9 +31,11 @@
  *                           all-reduce of a step fires its event as soon as all its CTAs have started, and the
  *                           next step's producers wait inside the kernel for its completion)
  *   SIFAR_PDL               0 = reducers are launched without programmatic dependent launch (read when the
- *                           library is loaded).  By default a reducer with more CTAs than the GPU has SMs
- *                           may become resident while the kernel before it on its stream drains; it reads
- *                           nothing until that kernel is complete.
+ *                           library is loaded).  By default a reducer with more CTAs than the GPU has SMs,
+ *                           or one whose producers were all enqueued on other streams, may become resident
+ *                           while the kernel before it on its stream drains.  In the two barrier-free modes
+ *                           its loads then start at once (they are ordered by flags or tags, not by the
+ *                           stream); everything it writes waits until that kernel is complete.
  *
  * All pointers named "device" are CUDA device pointers valid on the context's
  * device; "stream" arguments are cudaStream_t passed as void* (NULL = the legacy

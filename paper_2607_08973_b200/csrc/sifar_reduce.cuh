@@ -208,10 +208,13 @@ __device__ __forceinline__ bool sentinel_wait(const uint4 *const *src, size_t wa
            depending on where its polls happened to fall). */
         Deadline d;
         uint4 v0 = ld_slot(p);
+        if (!slot_valid(v0, e)) {                     /* already there (a thread's later units usually are): one look */
+        v0 = ld_slot(p);
         __nanosleep(kPollStaggerNs);
         uint4 v1 = ld_slot(p);
         __nanosleep(kPollStaggerNs);
         uint4 v2 = ld_slot(p);
+        ++reloads;
         for (;;) {
             if (slot_valid(v0, e)) break;
             v0 = ld_slot(p);
@@ -221,6 +224,7 @@ __device__ __forceinline__ bool sentinel_wait(const uint4 *const *src, size_t wa
             v2 = ld_slot(p);
             reloads += 3;
             if (d.expired(timeout_ns)) { ok = false; break; }
+        }
         }
     }
     return __all_sync(0xFFFFFFFFu, ok);
