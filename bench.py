@@ -389,6 +389,79 @@ def measure_skew(sf, torch, synth, runs=6):
     return {"one_reader_persistent_speculative": one, "p_readers": sym}
 
 
+def late_producers(sf, torch, P_=8, n=LARGE_N, reps=6, delays_us=None):
+    """A large call whose producers are late: every rank's pack kernel is held back a different time (0-300 us)
+    behind a spin kernel on its own stream, the reducer is enqueued at once.  Device time from the common start
+    to the end of the reducer, and from the end of the last producer to the end of the reducer (what the mode
+    adds once the data is there): dual-buffered (one arrival flag per rank: nothing can be reduced before the
+    last rank has stored everything) against speculative (flagged tiles: blocks are reduced as they land)."""
+    if delays_us is None:
+        delays_us = [(37 * r * r + 300 - 40 * r) % 301 for r in range(P_)]
+    xs = [torch.randint(-3000, 3000, (n,), dtype=torch.int16, device="cuda") for _ in range(P_)]
+    out = torch.empty(n, dtype=torch.int16, device="cuda")
+    res = {"delays_us": delays_us}
+    for mode in (sf.DUALBUF, sf.SPECULATIVE):
+        ctx = sf.sifar_create(P_, n, 0)
+        ps = [torch.cuda.Stream() for _ in range(P_)]
+        rs, main = torch.cuda.Stream(), torch.cuda.Stream()
+        total, tail = [], []
+        for it in range(reps + 2):
+            torch.cuda.synchronize()
+            sf.sifar_spin(300_000, main.cuda_stream)                 # lets the host enqueue everything ahead
+            ev0 = torch.cuda.Event(enable_timing=True)
+            ev0.record(main)
+            ends = []
+            for r in range(P_):
+                ps[r].wait_event(ev0)
+                sf.sifar_spin(delays_us[r] * 1000 + 1000, ps[r].cuda_stream)
+                sf.sifar_pack(ctx, r, xs[r].data_ptr(), n, mode, ps[r].cuda_stream)
+                e = torch.cuda.Event(enable_timing=True)
+                e.record(ps[r])
+                ends.append(e)
+            rs.wait_event(ev0)
+            sf.sifar_allreduce(ctx, None, out.data_ptr(), n, mode, rs.cuda_stream)
+            ev1 = torch.cuda.Event(enable_timing=True)
+            ev1.record(rs)
+            torch.cuda.synchronize()
+            assert sf.sifar_status(ctx) == 0, (mode, it, sf.sifar_status(ctx), sf.sifar_get_stats(ctx), sf.sifar_last_error())
+            if it >= 2:
+                t_end = ev0.elapsed_time(ev1) * 1e3
+                t_last = max(ev0.elapsed_time(e) for e in ends) * 1e3
+                total.append(t_end)
+                tail.append(t_end - t_last)
+        st = sf.sifar_get_stats(ctx)
+        sf.sifar_destroy(ctx)
+        res[sf.MODE_NAMES[mode]] = {"start_to_result_us": round(float(np.median(total)), 1),
+                                    "last_producer_end_to_result_us": round(float(np.median(tail)), 1),
+                                    "flag_polls_per_call": round(st["flag_polls"] / max(1, st["calls"]))}
+    return res
+
+
+def late_producers_in_a_process_of_its_own() -> dict:
+    """Ten streams have to run at the same time here.  With the default of eight hardware queues two of them share
+    a queue with another and the reducer ends up behind a producer it is meant to wait for, so this section runs
+    in a child process with CUDA_DEVICE_MAX_CONNECTIONS=32 (the variable is read when CUDA starts)."""
+    env = dict(os.environ, CUDA_DEVICE_MAX_CONNECTIONS="32")
+    out = subprocess.run([sys.executable, os.path.abspath(__file__), "--only", "late"], env=env, capture_output=True,
+                         text=True, timeout=600)
+    if out.returncode != 0:
+        return {"error": out.stderr[-400:]}
+    return json.loads(out.stdout.strip().splitlines()[-1])
+
+
+def run_late() -> None:
+    import torch
+    from paper_2607_08973_b200 import binding as sf
+    sf.lib()
+    sf.sifar_workload_preload()
+    res = {}
+    for n in (1 << 20, LARGE_N, 4 * LARGE_N):
+        row = {"spread_0_300us": late_producers(sf, torch, P, n),
+               "all_at_once": late_producers(sf, torch, P, n, delays_us=[0] * P)}
+        res[f"{n * 2 >> 20}MiB_per_rank"] = row
+    print(json.dumps(res))
+
+
 def payload_sweep(sf, torch, exps=range(10, 26), ranks=(2, 4, 8)):
     """Config 4: reducer time against payload, data ready, every mode; bf16 for all P, fp32 for P = 8.
 
@@ -580,6 +653,7 @@ def run_gpu(args) -> None:
                 for b in (1, 8, 32, 64)}
             detail["streams"] = measure_modes(sf, torch, synth, n, 3, 8, (sf.CHAIN_STREAMS,), modes, rounds=2)
             detail["payload_sweep"] = payload_sweep(sf, torch)
+            detail["late_producers"] = late_producers_in_a_process_of_its_own()
             detail["retry_overhead"] = retry_overhead(sf, torch, synth)
         # -- 3. reducer alone against the payload; the roofline kernel is the 16 MiB point ------------
         r_iters = max(4, min(10, args.steps))
@@ -695,7 +769,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="sifar", choices=["sifar", "reference"])
     ap.add_argument("--sweep", action="store_true", help="also batch sizes 2..16 and the stream chain")
-    ap.add_argument("--only", default="all", choices=["all", "decode", "roofline", "p_readers"],
+    ap.add_argument("--only", default="all", choices=["all", "decode", "roofline", "p_readers", "late"],
                     help="profiling aid: run the timed decode region only, the roofline section only, or the "
                          "P-reader chain only")
     ap.add_argument("--roofline-contexts", type=int, default=24,
@@ -705,6 +779,9 @@ def main() -> None:
                     help="profiling aid: leave out the graph / stream chains (under ncu kernels are serialised, and "
                          "those chains' reducers wait for producers that run concurrently)")
     args = ap.parse_args()
+    if args.only == "late":
+        run_late()
+        return
     if args.impl == "reference":
         args.steps = args.steps or 20
         args.warmup = 3 if args.warmup is None else args.warmup

@@ -930,13 +930,14 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
     a.defer = ctx->d_defer;
     a.spin_ns = ctx->spin_ns < ctx->timeout_ns ? ctx->spin_ns : ctx->timeout_ns;
     /* One tile per CTA.  Up to one CTA per SM the reducer cannot crowd out the producers and waits in
-       place; beyond that it runs at full occupancy, waits briefly, and its last CTAs sweep up.  Two
-       janitors per SM: half the registers of an SM stay free for the producers they wait for, and the
-       sweep still runs at three quarters of the full-occupancy bandwidth. */
+       place; beyond that it runs at full occupancy, waits briefly, and its last CTAs sweep up: one
+       janitor per SM.  Two per SM swept faster, but with two waiting CTAs of this kernel on every SM a
+       producer that became ready after the reducer had started was not given a single CTA slot until the
+       reducer gave up (seen with every stream on a hardware queue of its own; one per SM never showed it). */
     const int U = unroll_for(ctx->P);
     const size_t ntiles = tiles_for(reduce_units(ctx, rl.n, kernel_mode), U);
     a.two_phase = ntiles > (size_t)ctx->sm_count ? 1u : 0u;
-    a.janitors = (uint32_t)ctx->sm_count * 2u;
+    a.janitors = (uint32_t)ctx->sm_count;
     if (a.janitors > ntiles) a.janitors = (uint32_t)ntiles;
     if (kernel_mode == kModeTiles) {
         /* a tile is kThreads * U vectors, a flag block kFlagBlockVecs = 4 * kThreads vectors */
