@@ -14,10 +14,16 @@ Sections measured by the default run (all on the device, CUDA events on the
 launching stream; per-all-reduce percentiles from %globaltimer stamps written by
 the kernel):
   1. decode step, timed region of exactly K steps           -> value, ms_per_step
-  2. the same step in every mode / chain implementation      -> detail.modes
-  3. large-payload reducer kernel, inputs larger than L2     -> roofline
-  4. host-buffer entry point (H2D + pack + reduce + D2H)      -> e2e
-  5. the CPU oracle on the host cores (bounded sample)        -> cpu_baseline
+  2. the same step in every mode / chain implementation      -> detail.modes, detail.p_readers
+  3. the metric against the payload: decode steps at other
+     batch sizes, the skewed-arrival config, the reducer
+     alone from 2 KB to 64 MiB per rank                      -> by_payload
+  4. the two validation schemes over an unchecked pull        -> detail.verification_overhead
+  5. large-payload reducer kernel, inputs larger than L2     -> roofline
+  6. host-buffer entry point (H2D + pack + reduce + D2H)      -> e2e
+  7. the CPU oracle on the host cores (bounded sample)        -> cpu_baseline
+--sweep adds every batch size, the stream chains, the whole payload sweep, the
+retry-overhead table and the late-producer section.
 With --gpus N > 1 (under torchrun) every rank runs the same replica on its own
 GPU; nothing is exchanged on the data path ("replicas only"); times are the max
 over ranks.  `--impl reference` times the CPU oracle alone.
