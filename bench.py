@@ -16,14 +16,15 @@ the kernel):
   1. decode step, timed region of exactly K steps           -> value, ms_per_step
   2. the same step in every mode / chain implementation      -> detail.modes, detail.p_readers
   3. the metric against the payload: decode steps at other
-     batch sizes, the skewed-arrival config, the reducer
-     alone from 2 KB to 64 MiB per rank                      -> by_payload
+     batch sizes, the skewed-arrival config, a 16 MiB call
+     with late producers, the reducer alone from 2 KB to
+     64 MiB per rank                                         -> by_payload
   4. the two validation schemes over an unchecked pull        -> detail.verification_overhead
   5. large-payload reducer kernel, inputs larger than L2     -> roofline
   6. host-buffer entry point (H2D + pack + reduce + D2H)      -> e2e
   7. the CPU oracle on the host cores (bounded sample)        -> cpu_baseline
 --sweep adds every batch size, the stream chains, the whole payload sweep, the
-retry-overhead table and the late-producer section.
+retry-overhead table and the late-producer section at three sizes.
 With --gpus N > 1 (under torchrun) every rank runs the same replica on its own
 GPU; nothing is exchanged on the data path ("replicas only"); times are the max
 over ranks.  `--impl reference` times the CPU oracle alone.
@@ -255,8 +256,9 @@ def measure_modes(sf, torch, synth, n, warmup, reps, impls, modes, rounds=3, nam
 def measure_roofline(sf, torch, P_, n, mode, warmup, iters, dtype=0, nctx=24):
     """Device time per launch of the reducer kernel on payloads larger than L2.
 
-    `nctx` contexts are packed (untimed; every rank on its own producer stream, as in the protocol), then
-    their reducers run back to back between two CUDA events on the launching stream; every launch reads
+    `nctx` contexts are packed (untimed; every rank on its own producer stream, as in the protocol; the host
+    waits for them: a large call whose producers are still busy when it is enqueued gets a sweep kernel behind
+    its reducer, which `late_producers` measures), then their reducers run back to back between two CUDA events on the launching stream; every launch reads
     partials that the other launches' traffic (each larger than the 126 MB L2) has since evicted.  A spin
     kernel ahead of the first event lets the host enqueue the whole batch before the device reaches it, so
     host launch cost is not in the timed region.  A pair of events costs about 13 us of its own (start and
@@ -275,8 +277,7 @@ def measure_roofline(sf, torch, P_, n, mode, warmup, iters, dtype=0, nctx=24):
         for h in ctxs:
             for r in range(P_):
                 sf.sifar_pack(h, r, xs[r].data_ptr(), n, mode, ps[r].cuda_stream)
-        for r in range(P_):
-            s.wait_stream(ps[r])
+        torch.cuda.synchronize()      # data ready: no producer stream has work pending when the reducers are enqueued
         sf.sifar_spin(2_000_000, s.cuda_stream)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(s)
@@ -406,8 +407,10 @@ def late_producers(sf, torch, P_=8, n=LARGE_N, reps=6, delays_us=None):
     xs = [torch.randint(-3000, 3000, (n,), dtype=torch.int16, device="cuda") for _ in range(P_)]
     out = torch.empty(n, dtype=torch.int16, device="cuda")
     res = {"delays_us": delays_us}
-    for mode in (sf.DUALBUF, sf.SPECULATIVE):
+    for mode, policy in ((sf.DUALBUF, sf.SWEEP_AUTO), (sf.SPECULATIVE, sf.SWEEP_AUTO),
+                         (sf.DUALBUF, sf.SWEEP_NEVER), (sf.SPECULATIVE, sf.SWEEP_NEVER)):
         ctx = sf.sifar_create(P_, n, 0)
+        sf.sifar_debug_sweep_policy(ctx, policy)
         ps = [torch.cuda.Stream() for _ in range(P_)]
         rs, main = torch.cuda.Stream(), torch.cuda.Stream()
         total, tail = [], []
@@ -437,31 +440,32 @@ def late_producers(sf, torch, P_=8, n=LARGE_N, reps=6, delays_us=None):
                 tail.append(t_end - t_last)
         st = sf.sifar_get_stats(ctx)
         sf.sifar_destroy(ctx)
-        res[sf.MODE_NAMES[mode]] = {"start_to_result_us": round(float(np.median(total)), 1),
+        key = sf.MODE_NAMES[mode] + ("" if policy == sf.SWEEP_AUTO else "_swept_by_janitors")
+        res[key] = {"start_to_result_us": round(float(np.median(total)), 1),
                                     "last_producer_end_to_result_us": round(float(np.median(tail)), 1),
                                     "flag_polls_per_call": round(st["flag_polls"] / max(1, st["calls"]))}
     return res
 
 
-def late_producers_in_a_process_of_its_own() -> dict:
+def late_producers_in_a_process_of_its_own(which: str = "late") -> dict:
     """Ten streams have to run at the same time here.  With the default of eight hardware queues two of them share
     a queue with another and the reducer ends up behind a producer it is meant to wait for, so this section runs
     in a child process with CUDA_DEVICE_MAX_CONNECTIONS=32 (the variable is read when CUDA starts)."""
     env = dict(os.environ, CUDA_DEVICE_MAX_CONNECTIONS="32")
-    out = subprocess.run([sys.executable, os.path.abspath(__file__), "--only", "late"], env=env, capture_output=True,
+    out = subprocess.run([sys.executable, os.path.abspath(__file__), "--only", which], env=env, capture_output=True,
                          text=True, timeout=600)
     if out.returncode != 0:
         return {"error": out.stderr[-400:]}
     return json.loads(out.stdout.strip().splitlines()[-1])
 
 
-def run_late() -> None:
+def run_late(sizes=(1 << 20, LARGE_N, 4 * LARGE_N)) -> None:
     import torch
     from paper_2607_08973_b200 import binding as sf
     sf.lib()
     sf.sifar_workload_preload()
     res = {}
-    for n in (1 << 20, LARGE_N, 4 * LARGE_N):
+    for n in sizes:
         row = {"spread_0_300us": late_producers(sf, torch, P, n),
                "all_at_once": late_producers(sf, torch, P, n, delays_us=[0] * P)}
         res[f"{n * 2 >> 20}MiB_per_rank"] = row
@@ -641,6 +645,7 @@ def run_gpu(args) -> None:
                 by_payload["moe_step_by_batch_tokens"][str(b)] = measure_modes(
                     sf, torch, synth, HIDDEN * b, 3, 6, impls, modes, rounds=2, name="moe", steps=120)
             by_payload["skewed_arrival_config5"] = measure_skew(sf, torch, synth)
+            by_payload["late_producers"] = late_producers_in_a_process_of_its_own("late16")
             detail["verification_overhead"] = verification_overhead(sf, torch, synth)
         if args.sweep and args.only == "all":
             for P_ in (2, 4, 8):
@@ -775,7 +780,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="sifar", choices=["sifar", "reference"])
     ap.add_argument("--sweep", action="store_true", help="also batch sizes 2..16 and the stream chain")
-    ap.add_argument("--only", default="all", choices=["all", "decode", "roofline", "p_readers", "late"],
+    ap.add_argument("--only", default="all", choices=["all", "decode", "roofline", "p_readers", "late", "late16"],
                     help="profiling aid: run the timed decode region only, the roofline section only, or the "
                          "P-reader chain only")
     ap.add_argument("--roofline-contexts", type=int, default=24,
@@ -785,8 +790,8 @@ def main() -> None:
                     help="profiling aid: leave out the graph / stream chains (under ncu kernels are serialised, and "
                          "those chains' reducers wait for producers that run concurrently)")
     args = ap.parse_args()
-    if args.only == "late":
-        run_late()
+    if args.only in ("late", "late16"):
+        run_late() if args.only == "late" else run_late((LARGE_N,))
         return
     if args.impl == "reference":
         args.steps = args.steps or 20

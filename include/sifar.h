@@ -36,6 +36,8 @@
  *                           while the kernel before it on its stream drains.  In the two barrier-free modes
  *                           its loads then start at once (they are ordered by flags or tags, not by the
  *                           stream); everything it writes waits until that kernel is complete.
+ *   SIFAR_SWEEP             0 = contexts start with SIFAR_SWEEP_NEVER (see sifar_debug_sweep_policy; read when
+ *                           the library is loaded)
  *
  * All pointers named "device" are CUDA device pointers valid on the context's
  * device; "stream" arguments are cudaStream_t passed as void* (NULL = the legacy
@@ -160,6 +162,11 @@ int sifar_destroy(sifar_ctx *ctx);
  * a waiting reducer of more than about 64 CTAs (n > 98 304 bf16 at P = 8) kept the
  * producers off the SMs it occupied.  For payloads of that size enqueue the
  * reducer behind its producers (an event or a graph edge); nothing is lost there.
+ * Outside a graph, a call of at least 8 reducer tiles per SM (4.6 MiB per rank at
+ * P = 8) in plain format whose producers still have work pending on their own
+ * streams when this function is called is enqueued as two kernels, the reducer
+ * grid and a sweep kernel for the tiles that grid had to leave
+ * (sifar_debug_sweep_policy).
  */
 int sifar_allreduce(sifar_ctx *ctx, const void *const *rank_ptrs, void *out, size_t n,
                     int mode, void *stream);
@@ -284,6 +291,24 @@ int sifar_tile_flags(sifar_ctx *ctx, int rank, void **flags, size_t *elems_per_f
  * a persistent chain, and for stream / graph chains created afterwards.
  */
 int sifar_debug_force_retries(sifar_ctx *ctx, unsigned rounds);
+
+/*
+ * Measurement hook: who reduces the tiles that a large reducer grid had to queue because its producers
+ * were late (one-GPU emulation only: Section 3.5's early start, with the reducer and its producers
+ * sharing one machine; the paper's ranks each have a GPU of their own and no counterpart for this).
+ *   SIFAR_SWEEP_AUTO (default; SIFAR_SWEEP=0 in the environment makes NEVER the default): a call in plain
+ *     format (barrier modes, flagged tiles) of at least 8 tiles per SM whose P producers were all enqueued
+ *     with sifar_pack / sifar_arrive on streams other than the reducer's gets a sweep kernel of its own,
+ *     behind the reducer grid on the same stream, if at least one of those streams still has work pending
+ *     when sifar_allreduce is called (cudaStreamQuery); the grid then keeps no janitors.  Not while the
+ *     stream is being captured.  A stream handed to sifar_pack / sifar_arrive must therefore stay alive until
+ *     the sifar_allreduce of the same call number has returned.
+ *   SIFAR_SWEEP_NEVER: queued tiles are always swept by the grid's own last CTAs (one per SM).
+ *   SIFAR_SWEEP_ALWAYS: as AUTO without asking the streams (what the extra kernel costs on ready data).
+ * Results do not depend on it.  Takes effect for sifar_allreduce calls enqueued afterwards.
+ */
+enum sifar_sweep_policy { SIFAR_SWEEP_NEVER = 0, SIFAR_SWEEP_AUTO = 1, SIFAR_SWEEP_ALWAYS = 2 };
+int sifar_debug_sweep_policy(sifar_ctx *ctx, int policy);
 
 /*
  * All-reduce without any allocation.  The paper has no counterpart for this call.

@@ -54,6 +54,7 @@ def lib() -> ctypes.CDLL:
             "sifar_reset": (ci, [vp, vp]),
             "sifar_debug_set_epoch": (ci, [vp, cu]),
             "sifar_debug_force_retries": (ci, [vp, cu]),
+            "sifar_debug_sweep_policy": (ci, [vp, ci]),
             "sifar_spec_format": (ci, [ci, ci, sz]),
             "sifar_tile_flags": (ci, [vp, ci, ctypes.POINTER(vp), ctypes.POINTER(sz), ctypes.POINTER(sz)]),
             "sifar_slot_count": (sz, [ci, sz]),
@@ -162,6 +163,13 @@ def sifar_tile_flags(ctx: int, rank: int) -> tuple[int, int, int]:
 
 def sifar_debug_force_retries(ctx: int, rounds: int) -> int:
     return _check(lib().sifar_debug_force_retries(ctx, rounds))
+
+
+SWEEP_NEVER, SWEEP_AUTO, SWEEP_ALWAYS = 0, 1, 2
+
+
+def sifar_debug_sweep_policy(ctx: int, policy: int) -> int:
+    return _check(lib().sifar_debug_sweep_policy(ctx, policy))
 
 
 def sifar_slot_count(dtype: int, n: int) -> int:

@@ -89,6 +89,7 @@ struct ReduceArgs {
     uint32_t early;          /* 1: reads do not wait for the stream's previous kernel, writes do     */
     uint32_t e_host;         /* the call number the host expects, or 0: take it from device memory   */
     uint32_t pdl;            /* host side only: launch with programmatic stream serialization         */
+    uint32_t sweeper;        /* 1: k_sweep follows on the stream: this grid keeps no count and no janitors */
 };
 
 struct PackArgs {
@@ -145,6 +146,28 @@ __device__ __forceinline__ void publish_call(DevState *st, uint32_t e, int P)
  * or slots) and is reduced by one CTA: every thread issues its U * P coalesced
  * 16-byte loads before the first add.
  */
+/* Ragged tail of a plain partial (fewer elements than a 16-byte vector holds): one element per thread, with the
+   last tile. */
+template <int DT, int P>
+__device__ __forceinline__ void ragged_tail(const ReduceArgs &a)
+{
+    constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
+    const size_t i = (size_t)a.n / EPV * EPV + threadIdx.x;
+    if (i >= a.n) return;
+    uint32_t w[P];
+    if (DT == SIFAR_BF16) {
+#pragma unroll
+        for (int r = 0; r < P; ++r)
+            w[r] = ld_relaxed_u16(reinterpret_cast<const uint16_t *>(a.src[r]) + i);
+        reinterpret_cast<uint16_t *>(a.out)[i] = (uint16_t)(sum_word<DT, P>(w) & 0xFFFFu);
+    } else {
+#pragma unroll
+        for (int r = 0; r < P; ++r)
+            w[r] = ld_relaxed_u32(reinterpret_cast<const uint32_t *>(a.src[r]) + i);
+        reinterpret_cast<uint32_t *>(a.out)[i] = sum_word<DT, P>(w);
+    }
+}
+
 template <int DT, int P>
 __device__ __forceinline__ void tile_plain(const ReduceArgs &a, size_t tile, size_t ntiles, bool wait_before_stores)
 {
@@ -168,22 +191,7 @@ __device__ __forceinline__ void tile_plain(const ReduceArgs &a, size_t tile, siz
         const size_t v = base + (size_t)u * kThreads;
         if (v < nvec) out[v] = sum_vec<DT, P>(x[u], true);
     }
-    /* Ragged tail (fewer than EPV elements): one element per thread, with the last tile. */
-    const size_t i = nvec * EPV + threadIdx.x;
-    if (tile == ntiles - 1 && i < a.n) {
-        uint32_t w[P];
-        if (DT == SIFAR_BF16) {
-#pragma unroll
-            for (int r = 0; r < P; ++r)
-                w[r] = ld_relaxed_u16(reinterpret_cast<const uint16_t *>(a.src[r]) + i);
-            reinterpret_cast<uint16_t *>(a.out)[i] = (uint16_t)(sum_word<DT, P>(w) & 0xFFFFu);
-        } else {
-#pragma unroll
-            for (int r = 0; r < P; ++r)
-                w[r] = ld_relaxed_u32(reinterpret_cast<const uint32_t *>(a.src[r]) + i);
-            reinterpret_cast<uint32_t *>(a.out)[i] = sum_word<DT, P>(w);
-        }
-    }
+    if (tile == ntiles - 1) ragged_tail<DT, P>(a);
 }
 
 /* Returns false if a slot of this thread was still stale after `limit_ns`. */
@@ -499,11 +507,15 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a
         }
         /* the ranks are late: queue the tile and free the SM; the call number is still needed to arrive */
         if (threadIdx.x == 0) defer_tile(a, tile);
+        if (a.sweeper) return;
         e = entry_epoch(a, ld_relaxed_u32x2(&a.st->epoch));         /* after the wait: the predecessor has published */
         alive = (e != 0u);
     } else {
         tile_plain<DT, P>(a, tile, ntiles, a.early != 0u);             /* pull and reduce (phase 2) */
     }
+    /* a sweep kernel follows on the stream: it is ordered after this whole grid, reduces what was queued
+       and closes the call */
+    if (a.sweeper) return;
     /* phase 3 (bottom barrier, baseline only) and publication of the call number by the last CTA out */
     const Roles role = cta_arrive<MODE>(a, e, P, alive, false, tile);
     if (!role.janitor) return;
@@ -518,6 +530,130 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a
         if (alive) tile_plain<DT, P>(a, t, ntiles, false);
     }
     janitor_leave<MODE>(a, e, P, alive);
+}
+
+/*
+ * The sweep kernel: second half of a large call in plain format whose producers are still busy on other
+ * streams when the call is enqueued.
+ *
+ * The janitors of k_reduce_plain sweep queued tiles with the registers of one quarter-occupancy CTA per
+ * SM: P loads of 16 bytes per thread, 32 KB per SM in flight, a third of the machine's bandwidth (42 us
+ * for the 134 MB of a 16 MiB/rank call at P = 8).  Such a call gets this kernel behind its reducer grid
+ * instead, and the grid keeps neither a CTA count nor janitors.  One CTA per SM as well, so that the late
+ * producers find room beside it, but compiled for one CTA per SM: a thread keeps kSweepTiles tiles in flight
+ * (128 KB per SM; 28 us for the same sweep).  It starts when the reducer grid is over (griddepcontrol.wait:
+ * the queue is complete and visible).  Nothing queued: CTA 0 closes the call and that is all.  Otherwise a
+ * CTA takes kSweepTiles queue entries per round, warp 0 checks all their flags with one round trip
+ * (lane = (tile, rank)), the CTA reduces them, and the last CTA out closes the call.
+ *
+ * (The same sweep out of shared memory - two stages of three tiles filled with cp.async, 56 registers, so
+ * that its CTAs fit beside a full reducer grid - was built and measured: 36 us instead of 28, the producers
+ * beside it 40 us slower, and no cheaper on ready data, where what this kernel costs is its place in the
+ * stream's chain of dependent launches, 1.1-1.8 us per call.)
+ */
+constexpr int kSweepTiles = 4;
+constexpr int kSweepFromTilesPerSm = 8;      /* below 8 queued tiles per janitor the janitors are as fast */
+
+template <int DT, int P, int MODE>
+__global__ void __launch_bounds__(kThreads, 1) k_sweep(const ReduceArgs a)
+{
+    constexpr int U = Unroll<P>::value;
+    constexpr int K = kSweepTiles;
+    constexpr int EPV = (DT == SIFAR_BF16) ? 8 : 4;
+    static_assert(K * P <= 32, "one lane of warp 0 per (tile, rank)");
+    __shared__ uint32_t s_e, s_n, s_tile[K];
+    __shared__ int s_ok;
+    DevState *st = a.st;
+    gdc_launch_dependents();
+    gdc_wait();
+    if (threadIdx.x == 0) {
+        uint32_t e = entry_epoch(a, ld_relaxed_u32x2(&st->epoch));
+        if (e && a.e_host && e != a.e_host) { fail(st, a.host_status, SIFAR_ERR_EPOCH); e = 0u; }
+        s_e = e;
+        s_n = e ? ld_relaxed_u32(a.defer) : 0u;
+    }
+    __syncthreads();
+    const uint32_t e = s_e, ndefer = s_n;
+    if (e == 0u) return;
+    if (ndefer == 0u) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) publish_call<MODE>(st, e, P);
+        return;
+    }
+    const size_t nvec = (size_t)a.n / EPV;
+    const size_t ntiles = tiles_for(nvec, U);
+    uint4 *out = reinterpret_cast<uint4 *>(a.out);
+    bool alive = true, checked = false;
+    for (uint32_t g = blockIdx.x; (size_t)g * K < ndefer && alive; g += gridDim.x) {
+        const uint32_t first = g * K;
+        const int cnt = (ndefer - first < (uint32_t)K) ? (int)(ndefer - first) : K;
+        if (threadIdx.x < 32) {
+            const int lane = (int)threadIdx.x, j = lane / P, r = lane % P;
+            const bool mine = j < cnt;
+            const uint32_t t = mine ? ld_relaxed_u32(a.defer + 1u + first + (uint32_t)j) : 0u;
+            if (mine && r == 0) s_tile[j] = t;
+            int why = 0, polls = 0;
+            /* flagged tiles: the flags of every queued tile; barrier modes: the same P flags, once */
+            if (mine && (MODE == kModeTiles || !checked)) {
+                const uint32_t *fp = a.flags + (size_t)(t >> a.flag_shift) * kFlagStride + r;
+                if (ld_acquire_u32(fp) != e) {
+                    polls = wait_flag_eq(fp, e, a.timeout_ns);
+                    if (polls < 0) { why = 1; polls = 0; }
+                    polls += 1;
+                }
+            }
+            why = __reduce_max_sync(0xFFFFFFFFu, why);
+            polls = __reduce_add_sync(0xFFFFFFFFu, polls);
+            if (lane == 0) {
+                s_ok = !why;
+                if (polls) atomicAdd(&st->stats[kStatFlagPolls], (unsigned long long)polls);
+                if (why) fail(st, a.host_status, SIFAR_ERR_TIMEOUT);
+            }
+        }
+        __syncthreads();
+        alive = (s_ok != 0);
+        checked = true;
+        if (alive) {
+            uint4 x[K][U][P];
+#pragma unroll
+            for (int j = 0; j < K; ++j) {
+                if (j < cnt) {
+                    const size_t base = (size_t)s_tile[j] * kThreads * U + threadIdx.x;
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const size_t v = base + (size_t)u * kThreads;
+                        if (v < nvec) {
+#pragma unroll
+                            for (int r = 0; r < P; ++r) x[j][u][r] = ld_slot(a.src[r] + v);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < K; ++j) {
+                if (j < cnt) {
+                    const size_t base = (size_t)s_tile[j] * kThreads * U + threadIdx.x;
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const size_t v = base + (size_t)u * kThreads;
+                        if (v < nvec) out[v] = sum_vec<DT, P>(x[j][u], true);
+                    }
+                    if (s_tile[j] == ntiles - 1) ragged_tail<DT, P>(a);
+                }
+            }
+        }
+        __syncthreads();                                    /* s_tile and s_ok are written again next round */
+    }
+    if (!__syncthreads_and(alive)) return;
+    if (threadIdx.x == 0) {
+        const uint32_t left = atom_add_relaxed_u32(&st->janitor_done, 1u) + 1u;
+        if (left == gridDim.x) {
+            st_relaxed_u32(&st->janitor_done, 0u);
+            st_relaxed_u32(a.defer, 0u);
+            /* flagged tiles: a tile that had to be queued was not there at the first look (mis-speculation) */
+            if (MODE == kModeTiles) st_relaxed_u32(&st->retry_epoch, e);
+            publish_call<MODE>(st, e, P);
+        }
+    }
 }
 
 template <int DT, int P>
@@ -803,6 +939,8 @@ __global__ void k_set_epoch(DevState *st, uint32_t e) { st->epoch = e; st->cta_a
  * bandwidth is what counts.  SIFAR_PDL=0 launches the plain way.
  */
 static bool g_pdl = !(getenv("SIFAR_PDL") && atoi(getenv("SIFAR_PDL")) == 0);
+/* SIFAR_SWEEP=0: contexts start with SIFAR_SWEEP_NEVER (the janitors of the reducer grid sweep, as for small grids). */
+static bool g_sweep = !(getenv("SIFAR_SWEEP") && atoi(getenv("SIFAR_SWEEP")) == 0);
 
 static thread_local cudaEvent_t g_programmatic_event = nullptr;   /* set by launch_reduce around the launch */
 
@@ -831,6 +969,31 @@ static cudaError_t launch_k(K kernel, int grid, cudaStream_t s, const ReduceArgs
        slows the graph chains and the host path */
     cfg.attrs = at; cfg.numAttrs = (g_pdl && (a.two_phase || a.pdl)) ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
+template <int DT, int P>
+static cudaError_t launch_sweep_p(int mode, int grid, cudaStream_t s, const ReduceArgs &a)
+{
+    switch (mode) {
+    case SIFAR_BARRIER_ONESHOT: return launch_k(k_sweep<DT, P, SIFAR_BARRIER_ONESHOT>, grid, s, a);
+    case SIFAR_DUALBUF:         return launch_k(k_sweep<DT, P, SIFAR_DUALBUF>, grid, s, a);
+    default:                    return launch_k(k_sweep<DT, P, kModeTiles>, grid, s, a);
+    }
+}
+
+template <int DT>
+static cudaError_t launch_sweep_dt(int P, int mode, int grid, cudaStream_t s, const ReduceArgs &a)
+{
+    switch (P) {
+    case 1: return launch_sweep_p<DT, 1>(mode, grid, s, a);
+    case 2: return launch_sweep_p<DT, 2>(mode, grid, s, a);
+    case 3: return launch_sweep_p<DT, 3>(mode, grid, s, a);
+    case 4: return launch_sweep_p<DT, 4>(mode, grid, s, a);
+    case 5: return launch_sweep_p<DT, 5>(mode, grid, s, a);
+    case 6: return launch_sweep_p<DT, 6>(mode, grid, s, a);
+    case 7: return launch_sweep_p<DT, 7>(mode, grid, s, a);
+    default: return launch_sweep_p<DT, 8>(mode, grid, s, a);
+    }
 }
 
 template <int DT, int P>
@@ -958,10 +1121,30 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
     /* Early reads need programmatic launch to mean anything, and the baseline keeps the plain stream order. */
     a.pdl = (rl.early && g_pdl && !rl.programmatic_event) ? 1u : 0u;
     a.early = (a.pdl && rl.mode != SIFAR_BARRIER_ONESHOT) ? 1u : 0u;
+    /* Large plain-format call whose producers run on other streams and have not all finished: their data
+       may be late, and what the grid then queues is swept by a kernel of its own (see k_sweep) instead of
+       the grid's janitors.  Not while capturing (a stream may not be queried then, and a graph's replays
+       meet other conditions than its capture did). */
+    a.sweeper = 0u;
+    if (ctx->sweep_policy != SIFAR_SWEEP_NEVER && rl.early && a.e_host && !rl.programmatic_event &&
+        kernel_mode != SIFAR_SPECULATIVE && ntiles >= (size_t)kSweepFromTilesPerSm * (size_t)ctx->sm_count) {
+        if (ctx->sweep_policy == SIFAR_SWEEP_ALWAYS) a.sweeper = 1u;
+        for (int r = 0; r < ctx->P && !a.sweeper; ++r) {
+            const cudaError_t q = cudaStreamQuery(ctx->prod_stream[r]);
+            if (q == cudaErrorNotReady) a.sweeper = 1u;
+            if (q != cudaSuccess) cudaGetLastError();          /* "not ready" is an answer, not an error */
+        }
+    }
     g_programmatic_event = rl.programmatic_event;
     cudaError_t err = (ctx->dtype == SIFAR_BF16)
         ? launch_reduce_dt<SIFAR_BF16>(ctx->P, kernel_mode, (int)ntiles, stream, a)
         : launch_reduce_dt<SIFAR_F32>(ctx->P, kernel_mode, (int)ntiles, stream, a);
+    if (err == cudaSuccess && a.sweeper) {
+        const size_t groups = (ntiles + kSweepTiles - 1) / kSweepTiles;
+        const int grid = (int)(groups < (size_t)ctx->sm_count ? groups : (size_t)ctx->sm_count);
+        err = (ctx->dtype == SIFAR_BF16) ? launch_sweep_dt<SIFAR_BF16>(ctx->P, kernel_mode, grid, stream, a)
+                                         : launch_sweep_dt<SIFAR_F32>(ctx->P, kernel_mode, grid, stream, a);
+    }
     g_programmatic_event = nullptr;
     SIFAR_CUDA(err);
     return SIFAR_OK;
@@ -987,6 +1170,9 @@ static cudaError_t preload_reducers()
     if (e == cudaSuccess) e = preload(k_reduce_plain<DT, P, SIFAR_DUALBUF>);
     if (e == cudaSuccess) e = preload(k_reduce_plain<DT, P, kModeTiles>);
     if (e == cudaSuccess) e = preload(k_reduce_spec<DT, P>);
+    if (e == cudaSuccess) e = preload(k_sweep<DT, P, SIFAR_BARRIER_ONESHOT>);
+    if (e == cudaSuccess) e = preload(k_sweep<DT, P, SIFAR_DUALBUF>);
+    if (e == cudaSuccess) e = preload(k_sweep<DT, P, kModeTiles>);
     return e;
 }
 
@@ -1106,6 +1292,7 @@ extern "C" sifar_ctx *sifar_create(int P, size_t max_elems, int dtype)
     c->timeout_ns = 200000ull * 1000ull;
     c->poll_wide_max = 16384;
     c->spin_ns = 5000;
+    c->sweep_policy = g_sweep ? SIFAR_SWEEP_AUTO : SIFAR_SWEEP_NEVER;
     if (const char *env = getenv("SIFAR_SPIN_NS")) c->spin_ns = strtoull(env, nullptr, 10);
     c->poll_pace_min = 16384;
     c->poll_sentinel_min = 16384;
@@ -1434,6 +1621,17 @@ extern "C" int sifar_debug_set_epoch(sifar_ctx *c, unsigned calls_so_far)
     c->h_epoch = calls_so_far;
     c->last_mode0_epoch = 0;
     memset(c->prod_epoch, 0, sizeof c->prod_epoch);
+    return SIFAR_OK;
+}
+
+extern "C" int sifar_debug_sweep_policy(sifar_ctx *c, int policy)
+{
+    if (!c) { set_error("sifar_debug_sweep_policy: NULL context"); return SIFAR_ERR_INVALID; }
+    if (policy < SIFAR_SWEEP_NEVER || policy > SIFAR_SWEEP_ALWAYS) {
+        set_error("sifar_debug_sweep_policy: unknown policy %d", policy);
+        return SIFAR_ERR_INVALID;
+    }
+    c->sweep_policy = policy;
     return SIFAR_OK;
 }
 

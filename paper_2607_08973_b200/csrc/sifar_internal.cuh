@@ -95,6 +95,7 @@ struct sifar_ctx {
     size_t poll_pace_min;            /* ... paced polling above this many pairs                              */
     uint32_t poll_pace_ns;
     size_t poll_sentinel_min;        /* ... sentinel wait per warp above this many pairs (persistent chain) */
+    int sweep_policy;                /* SIFAR_SWEEP_*: when a large call gets a sweep kernel of its own        */
     uint32_t force_retries;          /* measurement knob: forced re-load rounds per slot (0 in normal use)    */
     /* what the host knows about the producers of the next call (sifar_pack / sifar_arrive record it) */
     uint32_t prod_epoch[SIFAR_MAX_RANKS];   /* call number the rank's producer was enqueued for (0: none)      */

@@ -67,6 +67,49 @@ def test_flagged_tiles_with_producers_up_to_300_us_late(oracle, P, n, dtype):
         assert st["calls_with_retry"] == 1 and st["flag_polls"] > 0 and st["timeouts"] == 0
 
 
+MODES = [sf.BARRIER_ONESHOT, sf.DUALBUF, sf.SPECULATIVE]
+
+
+@pytest.mark.parametrize("policy", [sf.SWEEP_NEVER, sf.SWEEP_AUTO, sf.SWEEP_ALWAYS])
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("P,dtype,n", [(8, BF16, (6 << 20) + 5), (3, F32, (4 << 20) + 3)])
+def test_queued_tiles_are_swept_by_the_janitors_or_by_the_sweep_kernel(oracle, mode, policy, P, dtype, n):
+    """A large call (more than 8 tiles per SM, ragged tail) whose producers are late, then one on ready data,
+    then a late one again: the same bits whoever sweeps the queued tiles, and the call numbers stay in step."""
+    with Ctx(P, n, dtype, timeout_us=2_000_000) as ctx:
+        sf.sifar_debug_sweep_policy(ctx.h, policy)
+        xs = synth.rank_inputs(P, n, dtype, 21 + policy, "uniform")
+        xd = [to_device(x) for x in xs]
+        ps = [torch.cuda.Stream() for _ in range(P)]
+        rs = torch.cuda.Stream()
+        for call, late in enumerate((True, False, True)):
+            out = empty_out(n, dtype)
+            torch.cuda.synchronize()
+            for r in range(P):
+                if late:
+                    sf.sifar_spin(100_000 + 30_000 * ((r * 5 + call) % P), ps[r].cuda_stream)
+                sf.sifar_pack(ctx.h, r, xd[(r + call) % P].data_ptr(), n, mode, ps[r].cuda_stream)
+            if not late:
+                torch.cuda.synchronize()
+            sf.sifar_allreduce(ctx.h, None, out.data_ptr(), n, mode, rs.cuda_stream)
+            torch.cuda.synchronize()
+            assert sf.sifar_status(ctx.h) == 0, (call, sf.sifar_last_error())
+            got, tail = out_to_numpy(out, n, dtype)
+            want = oracle.allreduce([xs[(r + call) % P] for r in range(P)], dtype)
+            assert_bits_equal(got, want, dtype, f"call {call}")
+            assert canary_ok(tail, dtype)
+        st = sf.sifar_get_stats(ctx.h)
+        assert st["epoch"] == 3 and st["calls"] == 3 and st["timeouts"] == 0
+        if mode == sf.SPECULATIVE:
+            assert st["calls_with_retry"] == 2       # the two late calls, not the one on ready data
+
+
+def test_sweep_policy_is_checked():
+    with Ctx(2, 1024, BF16) as ctx:
+        with pytest.raises(sf.SifarError):
+            sf.sifar_debug_sweep_policy(ctx.h, 3)
+
+
 def test_a_fused_producer_that_signals_block_by_block(oracle):
     """The caller's own kernel stores plain data and releases the block flags itself (sifar_tile_flags,
     device helper signal_block): first half of the blocks, a pause, then the rest."""
