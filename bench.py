@@ -645,7 +645,8 @@ def run_gpu(args) -> None:
                 by_payload["moe_step_by_batch_tokens"][str(b)] = measure_modes(
                     sf, torch, synth, HIDDEN * b, 3, 6, impls, modes, rounds=2, name="moe", steps=120)
             by_payload["skewed_arrival_config5"] = measure_skew(sf, torch, synth)
-            by_payload["late_producers"] = late_producers_in_a_process_of_its_own("late16")
+            if not args.skip_graph:       # its reducer waits for producers that run beside it, as the graph chains' do
+                by_payload["late_producers"] = late_producers_in_a_process_of_its_own("late16")
             detail["verification_overhead"] = verification_overhead(sf, torch, synth)
         if args.sweep and args.only == "all":
             for P_ in (2, 4, 8):
@@ -787,8 +788,8 @@ def main() -> None:
                     help="profiling aid: contexts (launches) per timed region of the reducer-alone section; a capture "
                          "under ncu wants few (each holds 0.6 GB at 16 MiB per rank)")
     ap.add_argument("--skip-graph", action="store_true",
-                    help="profiling aid: leave out the graph / stream chains (under ncu kernels are serialised, and "
-                         "those chains' reducers wait for producers that run concurrently)")
+                    help="profiling aid: leave out the graph / stream chains and the late-producer section (under ncu "
+                         "kernels are serialised, and their reducers wait for producers that run concurrently)")
     args = ap.parse_args()
     if args.only in ("late", "late16"):
         run_late() if args.only == "late" else run_late((LARGE_N,))
