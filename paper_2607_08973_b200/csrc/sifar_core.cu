@@ -496,6 +496,13 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a
             }
         }
     }
+    if (MODE == kModeTiles && a.early && threadIdx.x == 33u) {
+        /* and for the flags of the CTA that takes this CTA's place a wave from now: block flags are read once
+           each, so unlike the one arrival line of the barrier modes they are not in the L2 when asked for */
+        const size_t later = tile + 4u * (size_t)a.janitors;
+        if (later < gridDim.x)
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(a.flags + (later >> a.flag_shift) * kFlagStride));
+    }
     uint32_t e = top_barrier<P, MODE>(a, tile, a.two_phase ? a.spin_ns : a.timeout_ns, give_up, true);
     bool alive = true;
     if (e == 0u) {
