@@ -350,6 +350,9 @@ __device__ __forceinline__ uint32_t top_barrier(const ReduceArgs &a, size_t tile
  *   wait until everybody has arrived, split the queued tiles among themselves
  *   and reduce them with the full time limit.  With producers that are on time
  *   the queue is empty and the janitors cost a short wait at the very end.
+ *   Where the host appends the sweep kernel (a.sweeper, see k_sweep) there are no
+ *   janitors and no count: a CTA reduces or queues its tile and leaves, and the
+ *   sweep kernel, ordered behind the whole grid, does the rest.
  *
  * Either way the last CTA out publishes the call (publish_call).
  */
