@@ -484,10 +484,12 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a
     if (!a.early) gdc_wait();
     gdc_launch_dependents();
     int give_up = 0;
-    if (a.early && (threadIdx.x & 7u) == 0u) {
+    if (a.early && !a.sweeper && (threadIdx.x & 7u) == 0u) {
         /* While warp 0 makes its round trip for the flags, ask the L2 for the tile's lines (one thread per
            128-byte line).  A prefetch returns nothing to the thread, so it cannot deliver stale data: the
-           loads below still follow the flags, and the L2 is where the producers' stores arrive. */
+           loads below still follow the flags, and the L2 is where the producers' stores arrive.  Not where
+           the host saw the producers still busy (a.sweeper): a grid that runs ahead of its producers would
+           read every partial once for nothing, beside the very kernels that are storing them. */
         constexpr int EPVp = (DT == SIFAR_BF16) ? 8 : 4;
         const size_t nvec = (size_t)a.n / EPVp;
 #pragma unroll
@@ -499,7 +501,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a
             }
         }
     }
-    if (MODE == kModeTiles && a.early && threadIdx.x == 33u) {
+    if (MODE == kModeTiles && a.early && !a.sweeper && threadIdx.x == 33u) {
         /* and for the flags of the CTA that takes this CTA's place a wave from now: block flags are read once
            each, so unlike the one arrival line of the barrier modes they are not in the L2 when asked for */
         const size_t later = tile + 4u * (size_t)a.janitors;
@@ -563,6 +565,7 @@ __global__ void __launch_bounds__(kThreads, 4) k_reduce_plain(const ReduceArgs a
  */
 constexpr int kSweepTiles = 4;
 constexpr int kSweepFromTilesPerSm = 8;      /* below 8 queued tiles per janitor the janitors are as fast */
+constexpr unsigned long long kSweepSpinNs = 500;   /* how long a CTA of the grid before it waits for its tile */
 
 template <int DT, int P, int MODE>
 __global__ void __launch_bounds__(kThreads, 1) k_sweep(const ReduceArgs a)
@@ -1145,6 +1148,8 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
             if (q != cudaSuccess) cudaGetLastError();          /* "not ready" is an answer, not an error */
         }
     }
+    /* with the sweep kernel behind it the grid need not hold the machine for tiles that are not there yet */
+    if (a.sweeper && a.spin_ns > kSweepSpinNs) a.spin_ns = kSweepSpinNs;
     g_programmatic_event = rl.programmatic_event;
     cudaError_t err = (ctx->dtype == SIFAR_BF16)
         ? launch_reduce_dt<SIFAR_BF16>(ctx->P, kernel_mode, (int)ntiles, stream, a)
