@@ -27,6 +27,11 @@
  *   SIFAR_POLL_PACE_NS/_MIN sleep between polling rounds above _MIN pairs (0 = unpaced)
  *   SIFAR_POLL_SENTINEL_MIN persistent chain: above this many pairs a warp first waits on one slot per rank (16384)
  *   SIFAR_CHAIN_CLUSTER     0 = persistent chain without thread-block clusters
+ *   SIFAR_CHAIN_HANDOFF_MAX persistent chain: up to this many (unit, rank) pairs a result reaches the next step's
+ *                           producers in tagged 16-byte words that each thread polls for itself, above it through one
+ *                           ready flag per chunk (100000)
+ *   SIFAR_CHAIN_WIDE_MAX    persistent speculative chain with tagged hand-over: re-poll all stale ranks per round up to
+ *                           this many (slot, rank) pairs, wait on a sentinel slot above (50000)
  *   SIFAR_CHAIN_PDL         0 = stream / graph chains record the step events the plain way (by default the
  *                           all-reduce of a step fires its event as soon as all its CTAs have started, and the
  *                           next step's producers wait inside the kernel for its completion)

@@ -15,8 +15,10 @@
  *                                              t > 1: from out^{t-1});
  *   out^t = all-reduce(x_0^t .. x_{P-1}^t)  in the chain's mode.
  * Producers of step t are ordered after the all-reduce of step t-1 (they consume
- * its result: stream event, graph edge, or a ready flag inside the persistent
- * kernel) and are NOT ordered before the all-reduce of step t by anything but
+ * its result: stream event, graph edge, or, inside the persistent kernel, result
+ * words that carry the call number and are polled by the thread that needs them
+ * (one ready flag per chunk for large grids; the done flags of the bottom barrier
+ * with both barriers)) and are NOT ordered before the all-reduce of step t by anything but
  * the arrival flags / slot tags of the mode under test.
  *
  * Update rules (each product and the sum rounded separately, no fused
@@ -134,12 +136,14 @@ int sifar_chain_chunks(sifar_chain *chain);
  * for every step s of a run, 48 words (0 = not taken; %globaltimer nanoseconds
  * unless stated) written by the CTAs that own chunk 0:
  *   reducer, thread 0:  [0] enters the step      [1] arrival flags seen (speculative: its warp's slots valid)
- *                       [2] whole chunk reduced  [3] ready flag released
+ *                       [2] whole chunk reduced  [3] result handed over (every thread has stored its units;
+ *                                                    large grids: ready flag released)
  *                       [28] done flags released (BARRIER_ONESHOT)
  *                       [29] number of slot re-loads of thread 0 in this step (a count)
  *                       [30..37] end of its first eight re-poll rounds (speculative)
  *   reducer, lane 0 of warp w:   [38+w] the warp's slots validated (speculative)
- *   producer of rank r, thread 0: [4+3r] previous result's ready flag seen   [5+3r] stores issued
+ *   producer of rank r, thread 0: [4+3r] previous result taken (its first unit's word valid, or the chunk's
+ *                                          ready / done flag seen)             [5+3r] stores issued
  *                                 [6+3r] arrival flag released (barrier modes)
  *   producer of rank 0, lane 0 of warp w: [42+w] the warp's stores issued
  * If `phases` is not NULL the words of the last run (steps_per_run x 48) are copied
