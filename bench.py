@@ -634,10 +634,9 @@ def run_gpu(args) -> None:
             detail["modes"] = measure_modes(sf, torch, synth, n, args.warmup, reps, impls, modes)
             detail["no_allreduce_note"] = (
                 "the same chain with each rank's next operation fed from its own partial (Section 2.4): what the "
-                "producers cost.  In the persistent kernel they read their own stores back through the L2 behind a "
-                "CTA barrier with the generator on the critical path, while the speculative chain overlaps the "
-                "generator with its wait and takes the previous result from the word it polls; at decode payloads "
-                "the two come out level, so it is not a lower bound there")
+                "producers cost.  In the persistent kernel a rank hands its partial to itself in the tagged 16-byte "
+                "words that carry an all-reduce result to the next step's producers, so step minus this is what "
+                "the all-reduce adds")
             detail["p_readers"] = {"llama P=8 8KB": measure_symmetric(sf, torch, synth, P, n)}
             # -- 2b. the metric is a curve: the same step against the payload, in the default run ---
             by_payload = {

@@ -71,7 +71,8 @@ typedef enum {
 
 /* Fourth "mode", chains only: no all-reduce at all; each rank's next operation consumes its own
    partial (the paper's "feed the input of the all-reduce to the next operation" experiment, Section 2.4).
-   The producers' own cost; its results are not a sum. */
+   The producers' own cost (in the persistent kernel a rank hands its partial to itself the way an all-reduce
+   result reaches the next step's producers); its results are not a sum. */
 enum { SIFAR_CHAIN_NO_ALLREDUCE = 3 };
 
 /* Fifth "mode", sifar_symchain_create only: the twoshot baseline (reduce-scatter, barrier, all-gather;

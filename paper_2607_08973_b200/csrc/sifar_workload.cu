@@ -338,7 +338,10 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
     }
     ChunkFlags *cf = a.chunks + chunk;
     const size_t n = (size_t)a.n;
-    constexpr int EPU = (MODE == SIFAR_SPECULATIVE) ? ((DT == SIFAR_BF16) ? 6 : 3) : ((DT == SIFAR_BF16) ? 8 : 4);
+    /* 12-byte units where the unit travels with a tag in one 16-byte word (speculative slots; the chain without
+       all-reduce, whose ranks hand their partial over to themselves the same way), else 16-byte vectors */
+    constexpr bool kSlotUnits = (MODE == SIFAR_SPECULATIVE || MODE == kModeNoAllreduce);
+    constexpr int EPU = kSlotUnits ? ((DT == SIFAR_BF16) ? 6 : 3) : ((DT == SIFAR_BF16) ? 8 : 4);
     /* Whole warps of units: a warp of which only some lanes have a unit was measured up to 0.4 us per step slower
        (the ragged last chunk then set the pace of the whole result).  Units past the last element carry zeros;
        the rank buffers and the ring rows have room for them. */
@@ -367,8 +370,10 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
         char *ring_row = a.ring + (size_t)((t - 1u) % a.ring_len) * a.ring_stride;
 
         constexpr bool tagged = TAGGED;          /* form of the hand-over, see handoff_store (the host's choice by size) */
-        uint4 *ho_cur = a.handoff + (size_t)p * a.handoff_stride;                 /* this step's result */
-        const uint4 *ho_prev = a.handoff + (size_t)(p ^ 1u) * a.handoff_stride;   /* the step before */
+        /* hand-over words [parity][unit]; without all-reduce [parity][rank][unit]: every rank hands its partial to itself */
+        const size_t ho_sets = no_ar ? (size_t)P : 1u, ho_mine = no_ar ? (size_t)rank : 0u;
+        uint4 *ho_cur = a.handoff + ((size_t)p * ho_sets + ho_mine) * a.handoff_stride;                 /* this step's result */
+        const uint4 *ho_prev = a.handoff + ((size_t)(p ^ 1u) * ho_sets + ho_mine) * a.handoff_stride;   /* the step before */
         if (is_reducer) {
             /* ---------------- the pulling side ---------------- */
             SIFAR_TRACE(0);
@@ -464,7 +469,7 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
             }
         } else {
             /* ---------------- rank `rank`, chunk `chunk` of the next operation ---------------- */
-            constexpr int NW = (MODE == SIFAR_SPECULATIVE) ? 3 : 4;
+            constexpr int NW = kSlotUnits ? 3 : 4;
             constexpr int NE = NW * ((DT == SIFAR_BF16) ? 2 : 1);
             const Gen g = make_gen(a.w, rank, t);
             const bool first = (t == 1u);
@@ -488,7 +493,7 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
                 for (int q = 0; q < NE; ++q) s_z[k - 1u][q][threadIdx.x] = z[q];
             }
             const uint32_t delay_ns = gen_delay_ns(a.w, rank, t);
-            const bool by_flag = no_ar || !tagged;       /* thread 0 waits for the chunk, then everybody loads */
+            const bool by_flag = !no_ar && !tagged;      /* thread 0 waits for the chunk, then everybody loads */
             if (by_flag || MODE == SIFAR_BARRIER_ONESHOT) {
                 if (threadIdx.x == 0) {
                     bool ok = true;
@@ -497,17 +502,16 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
                            buffer.  It released the done flags after its result stores and a CTA barrier, so the
                            flag hands the result over as well. */
                         if (t > 1u) ok = wait_flag_or_fail<true>(&cf->done[rank], e - 1u, st, a.host_status, a.timeout_ns);
-                    } else if (!no_ar && !tagged && t > 1u) {
+                    } else if (t > 1u) {
                         ok = wait_flag_or_fail<true>(&cf->ready, e - 1u, st, a.host_status, a.timeout_ns);
                     }
-                    if (by_flag) { SIFAR_TRACE(4 + 3 * rank); if (ok) spin_ns(delay_ns); }
+                    if (by_flag) { SIFAR_TRACE(4 + 3 * rank); if (ok) spin_ns(delay_ns); }   /* else: after the first unit is taken */
                     s_ok = ok;
                 }
                 __syncthreads();
                 if (!s_ok) { alive = false; break; }
             }
-            const char *prev = no_ar ? a.plain + ((size_t)(p ^ 1u) * P + rank) * a.plain_stride
-                                     : a.ring + (size_t)((t + a.ring_len - 2u) % a.ring_len) * a.ring_stride;
+            const char *prev = a.ring + (size_t)((t + a.ring_len - 2u) % a.ring_len) * a.ring_stride;   /* flag form */
             /* The previous result of unit u: polled where the reducer hands it over (first step: none).  The rank's
                seeded delay (skewed-arrival workload) follows the first unit's arrival, before anything is stored. */
             const auto take_prev = [&](size_t u, uint32_t (&pw)[NW], bool with_delay) -> bool {
@@ -519,7 +523,9 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
                 return ok;
             };
             const auto store_unit = [&](size_t u, const uint32_t (&w)[NW]) {
-                if (MODE == SIFAR_SPECULATIVE) {
+                if (no_ar) {
+                    handoff_store<3>(ho_cur, u, make_uint4(w[0], w[1], w[2], 0u), e);      /* to itself, next step */
+                } else if (MODE == SIFAR_SPECULATIVE) {
                     store_slot(reinterpret_cast<uint4 *>(a.slots + ((size_t)p * P + rank) * a.slot_stride), u,
                                w[0], w[1], w[2], e);
                 } else {
@@ -532,7 +538,7 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
             if (unit0 < nunits) {
                 uint32_t w[NW];
                 if (by_flag) {
-                    unit_combine<DT, NW>(g, first, prev, unit0 * EPU, n, z0, w, no_ar ? 0 : n_io);
+                    unit_combine<DT, NW>(g, first, prev, unit0 * EPU, n, z0, w, n_io);
                 } else {
                     uint32_t pw[NW];
                     mine_ok = take_prev(unit0, pw, true);
@@ -553,7 +559,7 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
                     unit_noise<DT, NW>(g, first, u * EPU, n, z);
                 }
                 if (by_flag) {
-                    unit_combine<DT, NW>(g, first, prev, u * EPU, n, z, w, no_ar ? 0 : n_io);
+                    unit_combine<DT, NW>(g, first, prev, u * EPU, n, z, w, n_io);
                 } else {
                     uint32_t pw[NW];
                     mine_ok = take_prev(u, pw, false);
@@ -573,7 +579,7 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
                 if (threadIdx.x == 0) st_release_u32(&cf->arrive[p][rank], e);
                 SIFAR_TRACE(6 + 3 * rank);
             } else if (no_ar) {
-                __syncthreads();
+                if (!__syncthreads_and(alive)) { alive = false; break; }
                 if (stamper && threadIdx.x == 0) my_stamps[s + 1u] = globaltimer_ns();
             }
         }
@@ -896,8 +902,8 @@ static int chain_setup_persistent(sifar_chain *ch)
 {
     sifar_ctx *c = ch->ctx;
     const int roles = (ch->mode == kModeNoAllreduce) ? c->P : c->P + 1;
-    const size_t units = (ch->mode == SIFAR_SPECULATIVE) ? slots_for(c->dtype, ch->n)
-                                                         : (ch->n * elem_size(c->dtype) + 15) / 16;
+    const size_t units = (ch->mode == SIFAR_SPECULATIVE || ch->mode == kModeNoAllreduce)
+                             ? slots_for(c->dtype, ch->n) : (ch->n * elem_size(c->dtype) + 15) / 16;
     /* how a result reaches the next step's producers: tagged words up to kHandoffMaxPairs polling threads, the
        chunks' ready flags above (see handoff_store); with both barriers the done flags do it */
     size_t max_pairs = kHandoffMaxPairs;
@@ -951,11 +957,13 @@ static int chain_setup_persistent(sifar_chain *ch)
     SIFAR_CUDA(cudaMemset(ch->d_retry_steps, 0, sizeof(uint32_t) * ch->steps));
     /* the hand-over buffer (see handoff_store): one 16-byte word per 12-byte unit, two per 16-byte vector, whole
        warps of units, both parities; zero = tag 0 = never valid.  Large grids use the chunks' ready flags instead. */
-    if (ch->tagged) {
+    if (ch->tagged || ch->mode == kModeNoAllreduce) {
+        /* without all-reduce every rank hands its partial over to itself in the same words: P sets per parity */
         const size_t padded = (units + 31) / 32 * 32;
-        ch->handoff_stride = padded * (ch->mode == SIFAR_SPECULATIVE ? 1 : 2);
-        SIFAR_CUDA(cudaMalloc(&ch->d_handoff, 2 * ch->handoff_stride * sizeof(uint4)));
-        SIFAR_CUDA(cudaMemset(ch->d_handoff, 0, 2 * ch->handoff_stride * sizeof(uint4)));
+        const size_t sets = (ch->mode == kModeNoAllreduce) ? (size_t)c->P : 1;
+        ch->handoff_stride = padded * (ch->mode == SIFAR_DUALBUF ? 2 : 1);
+        SIFAR_CUDA(cudaMalloc(&ch->d_handoff, 2 * sets * ch->handoff_stride * sizeof(uint4)));
+        SIFAR_CUDA(cudaMemset(ch->d_handoff, 0, 2 * sets * ch->handoff_stride * sizeof(uint4)));
     }
     return SIFAR_OK;
 }
