@@ -264,12 +264,15 @@ struct PersistArgs {
  * do in the speculative mode: data and call number in one 16-byte store, validated by the reader, who polls the
  * unit it needs and nothing else - no CTA-wide barrier, no fence, no flag, no second round trip for the data.
  * The other form, one ready flag per chunk (barrier, release; acquire poll by thread 0, barrier, then the loads),
- * costs 0.5-1.0 us more per step at decode payloads in every mode; it is kept for large grids (more than
- * kHandoffMaxPairs polling threads), where eight times as many threads polling data lines as there are units
- * slowed the reducers' stores more than the flag costs (measured: 128 KB per rank 3.8 against 3.6 us, 512 KB per
- * rank 14.2 against 11.7 us mean).
- * NW = 3 result words (speculative mode: a 12-byte unit): {w0, w1, w2, tag}.  NW = 4 (a 16-byte vector of the
- * barrier modes): two stores {w0, tag, w1, tag}, {w2, tag, w3, tag}, each valid by itself.
+ * costs 0.3-1.0 us more per step at decode payloads in the two barrier-free modes; it is kept for large grids
+ * (more than kHandoffMaxPairs polling threads), where eight times as many threads polling data lines as there
+ * are units slowed the reducers' stores more than the flag costs (measured at P = 8: 256 KB per rank 7.8 against
+ * 7.3 us, 512 KB per rank 14.2 against 11.7 us mean).  With both barriers neither form is needed: the done flags
+ * of the bottom barrier follow the result stores.  The chain without all-reduce uses the words too: every rank
+ * hands its partial to itself.
+ * NW = 3 result words (a 12-byte unit: speculative mode, chain without all-reduce): {w0, w1, w2, tag}.  NW = 4
+ * (a 16-byte vector of the dual-buffered mode): two stores {w0, tag, w1, tag}, {w2, tag, w3, tag}, each valid by
+ * itself.
  */
 template <int NW>
 __device__ __forceinline__ void handoff_store(uint4 *base, size_t u, const uint4 &v, uint32_t tag)
