@@ -165,8 +165,25 @@ def test_modes_agree_bitwise_on_every_step(oracle):
             assert np.array_equal(got, ref), (impl, mode)
 
 
+@pytest.mark.parametrize("mode", [sf.DUALBUF, sf.SPECULATIVE])
+@pytest.mark.parametrize("n,steps,name,handoff_max", [(4096, 64, "llama", "0"), (16384 * 8 + 5, 24, "moe", "1000000000"),
+                                                      (4096 * 3 + 1, 64, "skew", "0")])
+def test_both_forms_of_the_result_hand_over_at_both_grid_sizes(oracle, monkeypatch, mode, n, steps, name, handoff_max):
+    """Inside the persistent kernel a result reaches the next step's producers in tagged words (small grids) or
+    by one ready flag per chunk (large grids); the size decides.  Here each form runs where the other is the
+    default: the flag form at a decode payload, the tagged words on a grid whose threads take two units per step."""
+    monkeypatch.setenv("SIFAR_CHAIN_HANDOFF_MAX", handoff_max)
+    P = 8
+    _, d = _workloads(name, P)
+    got, st = run_chain(P, n, BF16, d, mode, sf.CHAIN_PERSISTENT, steps, runs=2)
+    want = oracle.chain(_oracle_w(oracle, d), P, n, BF16, 2 * steps)
+    for t in range(2 * steps):
+        assert_bits_equal(got[t], want[t], BF16, f"step {t + 1}")
+    assert st["timeouts"] == 0 and st["calls"] == 2 * steps
+
+
 def test_no_allreduce_floor_runs():
-    """The timing floor without all-reduce runs in every implementation and leaves the call number alone."""
+    """The chain without all-reduce runs in every implementation and leaves the call number alone."""
     P, n, steps = 8, 4096, 64
     _, d = _workloads("llama", P)
     for impl in IMPLS:
