@@ -308,6 +308,7 @@ __device__ __forceinline__ bool handoff_wait(const uint4 *base, size_t u, uint32
 }
 
 constexpr size_t kHandoffMaxPairs = 100000;
+constexpr size_t kChainClusterMaxPairs = 50000;  /* one thread-block cluster per chunk up to here, see chain_setup_persistent */
 constexpr size_t kChainWideMaxPairs = 50000;    /* speculative chain with tagged hand-over: wide polling up to here, sentinel above */      /* (unit, rank) pairs up to which the result is handed over in tagged words */
 constexpr int kChainThreads = 128;
 constexpr int kPreUnits = 4;            /* units per producer thread, beyond its first, whose seeded half is computed before the wait */
@@ -925,10 +926,14 @@ static int chain_setup_persistent(sifar_chain *ch)
         C = (units + (size_t)kChainThreads * K - 1) / ((size_t)kChainThreads * K);
     }
     ch->K = K; ch->C = (uint32_t)C; ch->grid = (int)(C * roles);
-    /* One cluster per chunk if the device can hold all of them at once (set SIFAR_CHAIN_CLUSTER=0 for the flat layout). */
+    /* One cluster per chunk if the device can hold all of them at once, for grids up to kChainClusterMaxPairs
+       (unit, rank) pairs: keeping a chunk's traffic inside one GPC takes 0.2-0.3 us off a step at decode payloads
+       (P = 8, 8 KB: 1.79 against 1.98 us speculative, 3.58 against 3.87 us with both barriers); larger grids did
+       better spread over the machine (128 KB: 3.81 against 3.34 us; 256 KB: 7.1 against 6.0 us dual-buffered mean).
+       SIFAR_CHAIN_CLUSTER=0: never. */
     ch->clustered = false;
     const char *env_cluster = getenv("SIFAR_CHAIN_CLUSTER");
-    if (!(env_cluster && atoi(env_cluster) == 0) && roles <= 16) {
+    if (!(env_cluster && atoi(env_cluster) == 0) && roles <= 16 && units * (size_t)c->P <= kChainClusterMaxPairs) {
         const void *fn = chain_kernel(ch);
         cudaError_t err = cudaSuccess;
         if (roles > 8) err = cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
@@ -1085,6 +1090,7 @@ extern "C" int sifar_chain_run(sifar_chain *ch, void *stream)
         a.cs = ch->d_cs; a.chunks = ch->d_chunks; a.stamps = ch->d_stamps; a.retry_steps = ch->d_retry_steps;
         a.trace = ch->trace_on ? ch->d_trace : nullptr;
         a.handoff = ch->d_handoff; a.handoff_stride = ch->handoff_stride;
+        a.clustered = ch->clustered ? 1u : 0u;
         void *params[] = {&a};
         const void *fn = chain_kernel(ch, ch->trace_on != 0);
         if (ch->clustered) {
