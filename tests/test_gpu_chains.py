@@ -110,7 +110,7 @@ def test_config2_llama_shaped_decode_step(oracle, b, mode, impl):
 
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("mode", MODES)
-@pytest.mark.parametrize("b", [1, 64])
+@pytest.mark.parametrize("b", [1, 32, 64])
 def test_config3_moe_shaped_decode_step(oracle, b, mode, impl):
     P, n, steps = 8, 4096 * b, 120
     _, d = _workloads("moe", P)
