@@ -26,7 +26,8 @@
  *   SIFAR_POLL_WIDE_MAX     re-poll all stale ranks per round up to this many (slot, rank) pairs (16384)
  *   SIFAR_POLL_PACE_NS/_MIN sleep between polling rounds above _MIN pairs (0 = unpaced)
  *   SIFAR_POLL_SENTINEL_MIN persistent chain: above this many pairs a warp first waits on one slot per rank (16384)
- *   SIFAR_CHAIN_CLUSTER     0 = persistent chain without thread-block clusters
+ *   SIFAR_CHAIN_CLUSTER     0 = persistent chain without thread-block clusters (by default the CTAs of a chunk are
+ *                           one cluster, for placement, on grids of up to 50000 (unit, rank) pairs)
  *   SIFAR_CHAIN_HANDOFF_MAX persistent chain: up to this many (unit, rank) pairs a result reaches the next step's
  *                           producers in tagged 16-byte words that each thread polls for itself, above it through one
  *                           ready flag per chunk (100000)
