@@ -132,6 +132,16 @@ int sifar_chain_chunk_stamps(sifar_chain *chain, int chunk, unsigned long long *
 int sifar_chain_chunks(sifar_chain *chain);
 
 /*
+ * How a PERSISTENT chain is laid out, as the host chose it and as the kernel of the last run saw it (synchronizes
+ * the device): out[0] chunks, [1] units per thread and step, [2] CTAs, [3] 1 = the CTAs of a chunk are launched as
+ * one thread-block cluster, [4] 1 = results reach the next step's producers in tagged words (0 = ready flag per
+ * chunk, or done flags with both barriers); from the kernel: [5] the role layout it used (1 = clustered), [6] CTAs
+ * per cluster as the hardware reported them (1 without clusters), [7] the form of the hand-over it was built for.
+ * Before the first run [5..7] are 0.
+ */
+int sifar_chain_geometry(sifar_chain *chain, unsigned out[8]);
+
+/*
  * Phase timeline of the persistent chain (the latency breakdown that stands in for
  * a bandwidth figure at decode payloads).  enable != 0 makes later runs record,
  * for every step s of a run, 48 words (0 = not taken; %globaltimer nanoseconds

@@ -235,6 +235,7 @@ def _wl() -> ctypes.CDLL:
             "sifar_chain_stamps": (ci, [vp, ullp]),
             "sifar_chain_chunk_stamps": (ci, [vp, ci, ullp]),
             "sifar_chain_chunks": (ci, [vp]),
+            "sifar_chain_geometry": (ci, [vp, ctypes.POINTER(ctypes.c_uint)]),
             "sifar_chain_launches_per_run": (ci, [vp]),
             "sifar_chain_trace": (ci, [vp, ci, ullp]),
             "sifar_chain_destroy": (ci, [vp]),
@@ -295,6 +296,14 @@ def sifar_chain_chunk_stamps(chain: int, chunk: int, steps_per_run: int) -> list
 
 def sifar_chain_chunks(chain: int) -> int:
     return _wl().sifar_chain_chunks(chain)
+
+
+def sifar_chain_geometry(chain: int) -> dict:
+    out = (ctypes.c_uint * 8)()
+    _check(_wl().sifar_chain_geometry(chain, out))
+    keys = ("chunks", "units_per_thread", "ctas", "clustered", "tagged", "kernel_clustered", "kernel_cluster_ctas",
+            "kernel_tagged")
+    return dict(zip(keys, (int(x) for x in out)))
 
 
 def sifar_chain_trace(chain: int, enable: bool, steps_per_run: int = 0):

@@ -223,7 +223,9 @@ struct __align__(128) ChunkFlags {
 
 struct __align__(128) ChainDev {
     uint32_t exit_count;            /* CTAs that left the kernel (monotonic)                        */
-    uint32_t pad0[31];
+    uint32_t seen[3];               /* written by CTA 0 of the last run: role layout (1 = clustered), CTAs per
+                                       cluster as the hardware reports them, form of the hand-over (1 = tagged) */
+    uint32_t pad0[28];
 };
 
 struct PersistArgs {
@@ -356,6 +358,12 @@ __global__ void __launch_bounds__(kChainThreads, 6) k_chain(const PersistArgs a)
     __shared__ int s_retried[2];
     __shared__ float s_z[kPreUnits][8][kChainThreads];   /* producers: seeded halves computed ahead of the wait */
     if (threadIdx.x < 2) s_retried[threadIdx.x] = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        /* what this launch really runs with, for sifar_chain_geometry */
+        uint32_t cluster_ctas;
+        asm volatile("mov.u32 %0, %%cluster_nctaid.x;" : "=r"(cluster_ctas));
+        a.cs->seen[0] = a.clustered; a.cs->seen[1] = cluster_ctas; a.cs->seen[2] = TAGGED ? 1u : 0u;
+    }
     __syncthreads();
     unsigned reloads = 0;
     bool alive = true;
@@ -1161,6 +1169,21 @@ extern "C" int sifar_chain_chunk_stamps(sifar_chain *ch, int chunk, unsigned lon
 }
 
 extern "C" int sifar_chain_chunks(sifar_chain *ch) { return ch && ch->impl == SIFAR_CHAIN_PERSISTENT ? (int)ch->C : 0; }
+
+extern "C" int sifar_chain_geometry(sifar_chain *ch, unsigned out[8])
+{
+    if (!ch || ch->impl != SIFAR_CHAIN_PERSISTENT || !out) {
+        set_error("sifar_chain_geometry: needs a persistent chain");
+        return SIFAR_ERR_INVALID;
+    }
+    ChainDev h;
+    SIFAR_CUDA(cudaDeviceSynchronize());
+    SIFAR_CUDA(cudaMemcpy(&h, ch->d_cs, sizeof h, cudaMemcpyDeviceToHost));
+    out[0] = ch->C; out[1] = ch->K; out[2] = (unsigned)ch->grid;
+    out[3] = ch->clustered ? 1u : 0u; out[4] = ch->tagged ? 1u : 0u;
+    out[5] = h.seen[0]; out[6] = h.seen[1]; out[7] = h.seen[2];
+    return SIFAR_OK;
+}
 
 extern "C" int sifar_chain_trace(sifar_chain *ch, int enable, unsigned long long *phases)
 {

@@ -187,6 +187,29 @@ def test_both_forms_of_the_result_hand_over_at_both_grid_sizes(oracle, monkeypat
     assert st["timeouts"] == 0 and st["calls"] == 2 * steps
 
 
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("n,clustered,tagged_modes", [(4096, 1, (sf.DUALBUF, sf.SPECULATIVE)), (4096 * 16, 0, (sf.DUALBUF, sf.SPECULATIVE)),
+                                                      (4096 * 32, 0, ())])
+def test_the_kernel_runs_with_the_layout_the_host_chose(mode, n, clustered, tagged_modes):
+    """Small grids: one thread-block cluster per chunk and tagged hand-over words; larger ones spread out; the
+    largest by ready flag.  The kernel reports what it really ran with."""
+    P, steps = 8, 8
+    _, d = _workloads("llama", P)
+    with Ctx(P, n, BF16) as ctx:
+        ring, _ = _ring(n, BF16, steps)
+        ch = sf.sifar_chain_create(ctx.h, sf.make_workload(**d), n, mode, sf.CHAIN_PERSISTENT, ring.data_ptr(), steps, steps)
+        try:
+            sf.sifar_chain_run(ch, 0)
+            g = sf.sifar_chain_geometry(ch)
+        finally:
+            sf.sifar_chain_destroy(ch)
+        assert sf.sifar_status(ctx.h) == 0
+    assert g["clustered"] == clustered and g["kernel_clustered"] == clustered
+    assert g["kernel_cluster_ctas"] == (P + 1 if clustered else 1)
+    assert g["tagged"] == g["kernel_tagged"] == int(mode in tagged_modes)
+    assert g["ctas"] == g["chunks"] * (P + 1)
+
+
 def test_no_allreduce_floor_runs():
     """The chain without all-reduce runs in every implementation and leaves the call number alone."""
     P, n, steps = 8, 4096, 64
