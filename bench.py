@@ -24,7 +24,8 @@ the kernel):
   6. host-buffer entry point (H2D + pack + reduce + D2H)      -> e2e
   7. the CPU oracle on the host cores (bounded sample)        -> cpu_baseline
 --sweep adds every batch size, the stream chains, the whole payload sweep, the
-retry-overhead table and the late-producer section at three sizes.
+retry-overhead table, the late-producer section at three sizes and the two forms of
+the persistent chain's result hand-over.
 With --gpus N > 1 (under torchrun) every rank runs the same replica on its own
 GPU; nothing is exchanged on the data path ("replicas only"); times are the max
 over ranks.  `--impl reference` times the CPU oracle alone.
@@ -472,6 +473,27 @@ def run_late(sizes=(1 << 20, LARGE_N, 4 * LARGE_N)) -> None:
     print(json.dumps(res))
 
 
+def handover_forms(sf, torch, synth, batches=(1, 4, 8, 16)):
+    """Persistent chain, P = 8: the two ways a result reaches the next step's producers, in the same build.  The
+    library picks by size (tagged words up to 100 000 (unit, rank) pairs); SIFAR_CHAIN_HANDOFF_MAX, read when a
+    chain is created, forces one or the other."""
+    modes = (sf.DUALBUF, sf.SPECULATIVE)
+    res, saved = {}, os.environ.get("SIFAR_CHAIN_HANDOFF_MAX")
+    try:
+        for form, env in (("tagged_words", "1000000000"), ("ready_flag_per_chunk", "0")):
+            os.environ["SIFAR_CHAIN_HANDOFF_MAX"] = env
+            res[form] = {}
+            for b in batches:
+                r = measure_modes(sf, torch, synth, HIDDEN * b, 5, 10, (sf.CHAIN_PERSISTENT,), modes, rounds=2)
+                res[form][f"{8 * b}KB"] = {k.split("/")[1]: {"p50_us": v["p50_us"], "p99_us": v["p99_us"]} for k, v in r.items()}
+    finally:
+        if saved is None:
+            os.environ.pop("SIFAR_CHAIN_HANDOFF_MAX", None)
+        else:
+            os.environ["SIFAR_CHAIN_HANDOFF_MAX"] = saved
+    return res
+
+
 def payload_sweep(sf, torch, exps=range(10, 26), ranks=(2, 4, 8)):
     """Config 4: reducer time against payload, data ready, every mode; bf16 for all P, fp32 for P = 8.
 
@@ -671,6 +693,7 @@ def run_gpu(args) -> None:
             detail["streams"] = measure_modes(sf, torch, synth, n, 3, 8, (sf.CHAIN_STREAMS,), modes, rounds=2)
             detail["payload_sweep"] = payload_sweep(sf, torch)
             detail["late_producers"] = late_producers_in_a_process_of_its_own()
+            detail["result_handover_forms"] = handover_forms(sf, torch, synth)
             detail["retry_overhead"] = retry_overhead(sf, torch, synth)
         # -- 3. reducer alone against the payload; the roofline kernel is the 16 MiB point ------------
         r_iters = max(4, min(10, args.steps))
