@@ -1143,6 +1143,12 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
         kernel_mode != SIFAR_SPECULATIVE && ntiles >= (size_t)kSweepFromTilesPerSm * (size_t)ctx->sm_count) {
         if (ctx->sweep_policy == SIFAR_SWEEP_ALWAYS) a.sweeper = 1u;
         for (int r = 0; r < ctx->P && !a.sweeper; ++r) {
+            /* a stream that is being captured may not be queried (the capture would be invalidated) */
+            cudaStreamCaptureStatus cap = cudaStreamCaptureStatusActive;
+            if (cudaStreamIsCapturing(ctx->prod_stream[r], &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
+                cudaGetLastError();
+                continue;
+            }
             const cudaError_t q = cudaStreamQuery(ctx->prod_stream[r]);
             if (q == cudaErrorNotReady) a.sweeper = 1u;
             if (q != cudaSuccess) cudaGetLastError();          /* "not ready" is an answer, not an error */
