@@ -307,7 +307,7 @@ int sifar_debug_force_retries(sifar_ctx *ctx, unsigned rounds);
  *     with sifar_pack / sifar_arrive on streams other than the reducer's gets a sweep kernel of its own,
  *     behind the reducer grid on the same stream, if at least one of those streams still has work pending
  *     when sifar_allreduce is called (cudaStreamQuery); the grid then keeps no janitors.  Not while the
- *     stream is being captured.  A stream handed to sifar_pack / sifar_arrive must therefore stay alive until
+ *     stream is being captured (a producer stream that is being captured is not asked and counts as idle).  A stream handed to sifar_pack / sifar_arrive must therefore stay alive until
  *     the sifar_allreduce of the same call number has returned.
  *   SIFAR_SWEEP_NEVER: queued tiles are always swept by the grid's own last CTAs (one per SM).
  *   SIFAR_SWEEP_ALWAYS: as AUTO without asking the streams (what the extra kernel costs on ready data).
