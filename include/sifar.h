@@ -42,6 +42,9 @@
  *                           while the kernel before it on its stream drains.  In the two barrier-free modes
  *                           its loads then start at once (they are ordered by flags or tags, not by the
  *                           stream); everything it writes waits until that kernel is complete.
+ *   SIFAR_BARRIER_EARLY     1 = the loads of a BARRIER_ONESHOT reducer may start early as well (they are ordered by
+ *                           its arrival flags); off by default, the baseline keeps the conventional stream order
+ *                           (read when the library is loaded)
  *   SIFAR_SWEEP             0 = contexts start with SIFAR_SWEEP_NEVER (see sifar_debug_sweep_policy; read when
  *                           the library is loaded)
  *

@@ -952,6 +952,9 @@ __global__ void k_set_epoch(DevState *st, uint32_t e) { st->epoch = e; st->cta_a
  * bandwidth is what counts.  SIFAR_PDL=0 launches the plain way.
  */
 static bool g_pdl = !(getenv("SIFAR_PDL") && atoi(getenv("SIFAR_PDL")) == 0);
+/* SIFAR_BARRIER_EARLY=1: the baseline's reads may start early too (they are ordered by its arrival flags just as
+   well); off by default: the baseline stands for the conventional design, which orders everything by the stream. */
+static bool g_barrier_early = getenv("SIFAR_BARRIER_EARLY") && atoi(getenv("SIFAR_BARRIER_EARLY")) != 0;
 /* SIFAR_SWEEP=0: contexts start with SIFAR_SWEEP_NEVER (the janitors of the reducer grid sweep, as for small grids). */
 static bool g_sweep = !(getenv("SIFAR_SWEEP") && atoi(getenv("SIFAR_SWEEP")) == 0);
 
@@ -1133,7 +1136,7 @@ int launch_reduce(sifar_ctx *ctx, const ReduceLaunch &rl, cudaStream_t stream)
     }
     /* Early reads need programmatic launch to mean anything, and the baseline keeps the plain stream order. */
     a.pdl = (rl.early && g_pdl && !rl.programmatic_event) ? 1u : 0u;
-    a.early = (a.pdl && rl.mode != SIFAR_BARRIER_ONESHOT) ? 1u : 0u;
+    a.early = (a.pdl && (rl.mode != SIFAR_BARRIER_ONESHOT || g_barrier_early)) ? 1u : 0u;
     /* Large plain-format call whose producers run on other streams and have not all finished: their data
        may be late, and what the grid then queues is swept by a kernel of its own (see k_sweep) instead of
        the grid's janitors.  Not while capturing (a stream may not be queried then, and a graph's replays
