@@ -51,8 +51,8 @@ LARGE_N = 8 << 20                      # 16 MiB of bf16 per rank
 NOMINAL_GBS = 8000.0                   # the HBM3e figure the metric names
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the roofline kernel at LARGE_N, from the
 # ncu capture summarised in the file named below; refreshed whenever the reducer kernels change
-NCU_TRAFFIC = {"bytes": 144_710_912, "captured_at_commit": "55ac632",
-               "summary": "profiles/k_reduce_plain_bf16_P8_16MiB.md (134.30 MB read + 10.41 MB written, flagged tiles, the median of three captured launches)"}
+NCU_TRAFFIC = {"bytes": 147_380_224, "captured_at_commit": "6a27414",
+               "summary": "profiles/k_reduce_plain_bf16_P8_16MiB.md (134.28 MB read + 13.10 MB written, flagged tiles, the median of three captured launches)"}
 
 
 def read_peaks() -> tuple[float, str]:
