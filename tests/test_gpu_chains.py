@@ -6,7 +6,8 @@ import torch
 from paper_2607_08973_b200 import binding as sf
 from paper_2607_08973_b200 import synth
 
-from gpu_util import BF16, F32, MODES, Ctx, assert_bits_equal
+from gpu_util import (BF16, F32, MODES, Ctx, allreduce_via_pack, assert_bits_equal, empty_out, out_to_numpy,
+                      to_device)
 
 pytestmark = pytest.mark.gpu
 
@@ -208,6 +209,36 @@ def test_the_kernel_runs_with_the_layout_the_host_chose(mode, n, clustered, tagg
     assert g["kernel_cluster_ctas"] == (P + 1 if clustered else 1)
     assert g["tagged"] == g["kernel_tagged"] == int(mode in tagged_modes)
     assert g["ctas"] == g["chunks"] * (P + 1)
+
+
+@pytest.mark.parametrize("handoff_max", ["100000", "0"])
+@pytest.mark.parametrize("mode", MODES)
+def test_a_wait_that_runs_out_ends_the_persistent_chain_and_the_context_recovers(oracle, monkeypatch, mode, handoff_max):
+    """Ranks delayed by up to 1 ms against a 50 us limit: whoever waits gives up, the kernel ends by itself, the
+    status is sticky, and after a reset the context works again; with either form of the result hand-over."""
+    monkeypatch.setenv("SIFAR_CHAIN_HANDOFF_MAX", handoff_max)
+    P, n, steps = 4, 4096, 8
+    d = dict(synth.chain_workload("llama", P), delay_max_ns=1_000_000)
+    xs = synth.rank_inputs(P, n, BF16, seed=79, dist="uniform")
+    xs_dev = [to_device(x) for x in xs]
+    with Ctx(P, n, BF16, timeout_us=50) as ctx:
+        ring, _ = _ring(n, BF16, steps)
+        ch = sf.sifar_chain_create(ctx.h, sf.make_workload(**d), n, mode, sf.CHAIN_PERSISTENT, ring.data_ptr(), steps, steps)
+        sf.sifar_chain_run(ch, 0)
+        torch.cuda.synchronize()                                         # returns: every wait is bounded
+        assert sf.sifar_status(ctx.h) == sf.ERR_TIMEOUT
+        with pytest.raises(sf.SifarError) as ei:                         # refused: the status is sticky
+            sf.sifar_chain_run(ch, 0)
+        assert ei.value.code == sf.ERR_TIMEOUT
+        sf.sifar_chain_destroy(ch)
+        sf.sifar_reset(ctx.h, 0)
+        sf.sifar_set_timeout_us(ctx.h, 2_000_000)
+        assert sf.sifar_status(ctx.h) == 0
+        out = empty_out(n, BF16)
+        allreduce_via_pack(ctx, xs_dev, n, mode, out)
+        torch.cuda.synchronize()
+        assert sf.sifar_status(ctx.h) == 0
+        assert_bits_equal(out_to_numpy(out, n, BF16)[0], oracle.allreduce(xs, BF16), BF16, "after the reset")
 
 
 def test_no_allreduce_floor_runs():
