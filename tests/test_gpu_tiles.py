@@ -104,6 +104,41 @@ def test_queued_tiles_are_swept_by_the_janitors_or_by_the_sweep_kernel(oracle, m
             assert st["calls_with_retry"] == 2       # the two late calls, not the one on ready data
 
 
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("policy", [sf.SWEEP_NEVER, sf.SWEEP_AUTO])
+def test_a_rank_that_is_too_late_for_a_large_call_times_out_and_the_context_recovers(oracle, mode, policy):
+    """One rank's producer is held back 20 ms against a 2 ms limit: the janitors, or the sweep kernel, give up
+    after the limit, the kernels end by themselves, the late producer finds the context dead and leaves, and
+    after a reset the same call works."""
+    P, dtype, n = 4, BF16, (5 << 20) + 3
+    with Ctx(P, n, dtype, timeout_us=2000) as ctx:
+        sf.sifar_debug_sweep_policy(ctx.h, policy)
+        xs = synth.rank_inputs(P, n, dtype, 31, "uniform")
+        xd = [to_device(x) for x in xs]
+        out = empty_out(n, dtype)
+        ps = [torch.cuda.Stream() for _ in range(P)]
+        rs = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        sf.sifar_spin(20_000_000, ps[P - 1].cuda_stream)                 # rank P-1: 20 ms late
+        for r in range(P):
+            sf.sifar_pack(ctx.h, r, xd[r].data_ptr(), n, mode, ps[r].cuda_stream)
+        sf.sifar_allreduce(ctx.h, None, out.data_ptr(), n, mode, rs.cuda_stream)
+        torch.cuda.synchronize()                                         # returns: every wait is bounded
+        assert sf.sifar_status(ctx.h) == sf.ERR_TIMEOUT
+        assert sf.sifar_get_stats(ctx.h)["timeouts"] >= 1
+        sf.sifar_reset(ctx.h, 0)
+        sf.sifar_set_timeout_us(ctx.h, 2_000_000)
+        assert sf.sifar_status(ctx.h) == 0
+        for r in range(P):
+            sf.sifar_pack(ctx.h, r, xd[r].data_ptr(), n, mode, ps[r].cuda_stream)
+        sf.sifar_allreduce(ctx.h, None, out.data_ptr(), n, mode, rs.cuda_stream)
+        torch.cuda.synchronize()
+        assert sf.sifar_status(ctx.h) == 0
+        got, tail = out_to_numpy(out, n, dtype)
+        assert_bits_equal(got, oracle.allreduce(xs, dtype), dtype, "after the reset")
+        assert canary_ok(tail, dtype)
+
+
 def test_sweep_policy_is_checked():
     with Ctx(2, 1024, BF16) as ctx:
         with pytest.raises(sf.SifarError):
